@@ -1,0 +1,194 @@
+/*
+ * kvb.h -- C ABI of libkvb: stitching independently cached KV chunks into one
+ * request's KV buffer, and choosing and attending the tokens to recompute.
+ *
+ * All entry points are plain C.  "device" pointers are CUDA global-memory
+ * addresses on the context's GPU and are owned by the caller; "host" pointers
+ * are ordinary process memory.  Tables passed by host pointer are consumed
+ * (copied) before the call returns.  The three data-path calls are
+ * asynchronous on the CUDA stream given (a cudaStream_t passed as void*), do
+ * not synchronise, and allocate nothing: the only allocations happen in
+ * kvb_create.  All calls on one context must be issued to one stream (or be
+ * ordered by the caller), because they share the context's descriptor arena
+ * and scratch.
+ *
+ * Errors: every call returns a kvb_status.  Tables are checked on the host
+ * before anything is launched; a rejected call launches nothing.  Device code
+ * never traps: a kernel that meets something it cannot process skips it and
+ * sets a sticky status word that kvb_last_status reads back.
+ *
+ * Tensor layouts (row-major, last index fastest; L layers, H = Hkv KV heads,
+ * d head_dim, T prompt tokens, C chunk_tokens):
+ *   KV buffer / fresh tensor  [L][2][T][H][d]  16-bit (bf16 or fp16), 0 = keys, 1 = values
+ *                             -- the prefill KV tensor shape of the paper's
+ *                             "Transformer KV Cache" section
+ *   cached chunk, keys/values INT8: [L][C][H][d] u8 codes
+ *                             INT4: [L][C][H][d/2] bytes, channel 2i in the low
+ *                                   nibble and 2i+1 in the high nibble of byte i
+ *                             FP16: [L][C][H][d] in the buffer's 16-bit dtype
+ *   key metadata              [L][G_k][H][d][2] float32 (scale, min); statistics per
+ *                             channel over a token group: G_k = 1 for INT8 (the whole
+ *                             chunk), C/int4_group for INT4
+ *   value metadata            [L][C][H][G_v][2] float32 (scale, min); statistics per token
+ *                             over a channel group: G_v = 1 for INT8, d/int4_group for INT4
+ * Cached keys are stored already rotated (RoPE) at absolute positions
+ * orig_pos .. orig_pos+C-1, as a prefill pass leaves them.
+ */
+#ifndef KVB_H_
+#define KVB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvb_ctx kvb_ctx; /* opaque */
+
+typedef enum {
+  KVB_OK = 0,
+  KVB_ERR_INVALID_ARG = 1,   /* NULL pointer, negative size, bad enum */
+  KVB_ERR_BAD_TABLE = 2,     /* chunk table does not tile [0,T), misaligned pointer, bad position */
+  KVB_ERR_UNSUPPORTED = 3,   /* shape or size outside what the kernels are built for */
+  KVB_ERR_WORKSPACE = 4,     /* call exceeds the limits given to kvb_create */
+  KVB_ERR_CUDA = 5,          /* a CUDA runtime call failed (kvb_last_error has the text) */
+  KVB_ERR_DEVICE_STATUS = 6, /* a kernel reported a problem (sticky) */
+  KVB_ERR_NO_DEVICE = 7      /* no usable sm_100 GPU */
+} kvb_status;
+
+typedef enum {
+  KVB_MODE_FRESH = 0, /* not cached: rows are taken bit for bit from the request's fresh tensor */
+  KVB_MODE_FP16 = 1,  /* cached, unquantised, in the buffer's 16-bit dtype */
+  KVB_MODE_INT8 = 2,
+  KVB_MODE_INT4 = 3
+} kvb_mode;
+
+/* Outcome of the lookup cascade (EXACT via prefix hash, APPROX via content hash, MISS). */
+typedef enum { KVB_MATCH_MISS = 0, KVB_MATCH_EXACT = 1, KVB_MATCH_APPROX = 2 } kvb_match;
+
+typedef enum { KVB_DT_F16 = 0, KVB_DT_BF16 = 1 } kvb_dtype;
+
+/* One row of a request's chunk table (host memory).  Mirrors the cached-chunk
+ * record of the paper's implementation section: both hashes, the absolute
+ * position the chunk was cached at, and where it goes in this prompt. */
+typedef struct {
+  uint8_t content_hash[32]; /* SHA-256 of the token ids (Dual-Hash Keying, Eq. 5); opaque here */
+  uint8_t prefix_hash[32];  /* chained SHA-256 (Eq. 4); opaque here */
+  int32_t orig_pos;         /* absolute position of the chunk's first token when it was cached */
+  int32_t new_pos;          /* position of its first token in this prompt */
+  int32_t n_tokens;         /* must equal the model's chunk_tokens */
+  int32_t mode;             /* kvb_mode */
+  int32_t match;            /* kvb_match; EXACT requires orig_pos == new_pos */
+  int32_t reserved;
+  const void* k_codes;      /* device; NULL for FRESH */
+  const void* v_codes;      /* device; NULL for FRESH */
+  const void* k_meta;       /* device; INT8 / INT4 only */
+  const void* v_meta;       /* device; INT8 / INT4 only */
+} kvb_chunk;
+
+/* One request.  Its chunks, sorted by new_pos, must tile [0, T) exactly. */
+typedef struct {
+  int32_t T;
+  int32_t n_chunks;
+  const kvb_chunk* chunks; /* host */
+  void* kv_buf;            /* device, [L][2][T][H][d], written by kvb_assemble */
+  const void* fresh;       /* device, same shape and dtype: freshly projected K~, V~ of every position */
+} kvb_request;
+
+typedef struct {
+  int32_t L, Hq, Hkv, d;
+  int32_t chunk_tokens;    /* C */
+  int32_t kv_dtype;        /* kvb_dtype of the KV buffer, the fresh tensor, FP16-mode chunks, Q and O */
+  int32_t int4_group;      /* tokens per key group and channels per value group in INT4 mode */
+  int32_t reserved;
+  double rope_theta;
+} kvb_model_desc;
+
+/* Upper bounds for ONE call; they size what kvb_create allocates. */
+typedef struct {
+  int32_t max_requests;
+  int32_t max_chunks_total;
+  int64_t max_tokens_total;
+} kvb_limits;
+
+typedef struct {
+  double ratio;        /* rho: k = floor(ratio * T) */
+  int32_t k_override;  /* >= 0: use this k instead */
+  int32_t seam_before; /* R of Algorithm 1: window [p-before, p+after) around each seam p */
+  int32_t seam_after;
+  int32_t which;       /* bit 0: keys (the printed deviation formula); bit 1: values */
+} kvb_select_params;
+
+/* Per-request outputs of the selection (device memory, caller-owned). */
+typedef struct {
+  float* delta;         /* [T]  cosine deviation of every position */
+  int32_t* rank;        /* [k]  the k most deviated positions, most deviated first (ties: lower index) */
+  int32_t* sel;         /* [sel_capacity] ascending union of rank[0..k) and the seam windows */
+  int32_t* n_sel;       /* [1]  number of valid entries of sel */
+  int32_t sel_capacity; /* >= k + seam tokens, or T */
+  int32_t reserved;
+} kvb_selection;
+
+/* Creates a context on `device` (a CUDA ordinal).  Allocates the descriptor
+ * arena (pinned host + device) and the deviation scratch for the given limits. */
+int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb_limits* limits);
+int kvb_destroy(kvb_ctx* ctx);
+
+/* Prompt Assembly, CHUNK_REUSE mode, with the steps the paper places before it
+ * fused in: for every cached chunk, dequantise (inverse of KV Quantization
+ * Eq. 6: x = code*scale + min; keys per channel, values per token), rotate the
+ * keys by R_theta^(new_pos - orig_pos) (the correction the Rotary Positional
+ * Embeddings section calls for; values are not rotated), and write rows
+ * new_pos .. new_pos+C-1 of every layer of kv_buf.  FRESH chunks copy the
+ * rows of `fresh`.  reqs: host array of n_req requests. */
+int kvb_assemble(kvb_ctx* ctx, const kvb_request* reqs, int n_req, void* cuda_stream);
+
+/* CacheBlendRecompute (Algorithm 2) steps 2 and 3 plus the token set of
+ * SelectiveRecompute (Algorithm 1):
+ *   delta_t = 1 - mean over layers, KV heads (and K/V per `which`) of
+ *             cos(kv_buf row, fresh row);
+ *   rank    = the floor(ratio*T) largest delta_t, ties broken by lower index;
+ *   sel     = ascending union of rank and [p-before, p+after) for every seam p
+ *             (an interior chunk boundary with a cached chunk on either side).
+ * out: host array of n_req kvb_selection (device pointers inside). */
+int kvb_deviation_topk(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_select_params* params,
+                       const kvb_selection* out, void* cuda_stream);
+
+/* Causal attention (Eq. 2) of the selected rows only.  q[r], out[r]: device,
+ * [L][sel_capacity][Hq][d] in kv_dtype; row i belongs to position sel[i] and
+ * attends keys 0..sel[i] of kv_buf; query head hq reads KV head hq/(Hq/Hkv).
+ * Rows >= *n_sel are left untouched.  softmax in float32. */
+int kvb_selective_attn(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_selection* sel,
+                       const void* const* q, void* const* out, float softmax_scale, void* cuda_stream);
+
+/* KV Quantization, Eq. 6 (cache-population side), for one chunk: x [L][C][H][d]
+ * in kv_dtype (device) -> codes and (scale, min) metadata in the layouts above.
+ * is_value = 0: keys, per channel; 1: values, per token.  bits: 4 or 8. */
+int kvb_quantize_chunk(kvb_ctx* ctx, const void* x, int is_value, int bits, void* codes, void* meta,
+                       void* cuda_stream);
+
+/* Host-only: runs the table checks the data-path calls run before launching
+ * (chunks in prompt order tiling [0,T), enums, positions, pointer alignment,
+ * the limits) without touching a GPU.  need_payload != 0 also requires the
+ * code / metadata pointers, as kvb_assemble does.  err (optional) receives
+ * the message.  No counterpart in the paper: it is the guard that keeps a bad
+ * table from ever reaching a kernel. */
+int kvb_validate(const kvb_model_desc* model, const kvb_limits* limits, const kvb_request* reqs, int n_req,
+                 int need_payload, char* err, size_t err_len);
+
+/* floor(ratio * T), the k of Algorithm 2 step 3. */
+int kvb_select_count(int T, double ratio);
+
+/* Synchronises the context's last stream and returns the sticky device status (0 = clean). */
+int kvb_last_status(kvb_ctx* ctx);
+/* Text of the last host-side error of this context (valid until the next call). */
+const char* kvb_last_error(kvb_ctx* ctx);
+const char* kvb_status_string(int status);
+/* Number of kernels this context has launched so far. */
+int64_t kvb_launch_count(kvb_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVB_H_ */

@@ -246,18 +246,18 @@ void kvo_dequant_v(const uint8_t* codes, const float* meta, int C, int H, int d,
  * f_j = theta^(-2j/d), angle delta * f_j, all in double. */
 void kvo_rope_rotate(double* rows, int64_t n, int H, int d, double theta, double delta) {
   int half = d / 2;
-  for (int64_t t = 0; t < n; t++)
-    for (int h = 0; h < H; h++) {
-      double* v = rows + (t * H + h) * d;
-      for (int j = 0; j < half; j++) {
-        double f = pow(theta, -2.0 * (double)j / (double)d);
-        double a = delta * f;
-        double c = cos(a), s = sin(a);
+  for (int j = 0; j < half; j++) {
+    double f = pow(theta, -2.0 * (double)j / (double)d);
+    double a = delta * f;
+    double c = cos(a), s = sin(a);
+    for (int64_t t = 0; t < n; t++)
+      for (int h = 0; h < H; h++) {
+        double* v = rows + (t * H + h) * d;
         double lo = v[j], hi = v[j + half];
         v[j] = lo * c - hi * s;
         v[j + half] = hi * c + lo * s;
       }
-    }
+  }
 }
 
 /* ------------------------------------------------------------------ */

@@ -1,0 +1,387 @@
+// Stitching kernel: dequantise (inverse of KV Quantization Eq. 6), rotate keys by
+// R_theta^(new_pos - orig_pos) (Rotary Positional Embeddings, Eq. 3) and write the rows
+// of one cached chunk into the request's [L][2][T][H][d] buffer (Prompt Assembly).
+//
+// One CTA per (chunk, layer, K|V).  The chunk-layer's packed codes and its (scale, min)
+// metadata are contiguous in global memory, so one thread fetches them with bulk async
+// copies (TMA, mbarrier completion) in four parts; half-warps start on a part as soon as it
+// lands.  A half-warp owns one KV head and a run of tokens; lane ln owns channels
+// 4ln..4ln+3 and their rotation partners 64+4ln..64+4ln+3, so both operands of every
+// rotation pair sit in the same thread and the per-channel affine terms
+//     k'_c = A_c q_c + B_c q_(c^64) + C_c
+// (scale, min, cos and sin folded together once per token group) stay in registers.
+// Output rows go out as 128-byte contiguous stores per half-warp.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "kvb_internal.h"
+
+namespace kvb {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kParts = 4;
+constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr int kHeadDim = 128;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after kWaitLimit polls (never expected; keeps a bad launch from hanging).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 64) __nanosleep(64);
+  }
+  return false;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+// byte k of x -> float, exactly: place it in the mantissa of 2^23 and subtract 2^23
+template <int K>
+__device__ __forceinline__ float byte_to_float(uint32_t x) {
+  return __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650u + K)) - 8388608.0f;
+}
+template <int K>
+__device__ __forceinline__ float nibble_to_float(uint32_t x) {
+  return __uint_as_float(((x >> (4 * K)) & 0xFu) | 0x4B000000u) - 8388608.0f;
+}
+
+template <typename T>
+struct Pack;
+template <>
+struct Pack<__nv_bfloat16> {
+  static __device__ __forceinline__ uint32_t two(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+  }
+  static __device__ __forceinline__ float2 unpack(uint32_t x) {
+    return make_float2(__uint_as_float(x << 16), __uint_as_float(x & 0xFFFF0000u));
+  }
+};
+template <>
+struct Pack<__half> {
+  static __device__ __forceinline__ uint32_t two(float a, float b) {
+    __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+  }
+  static __device__ __forceinline__ float2 unpack(uint32_t x) {
+    return __half22float2(*reinterpret_cast<__half2*>(&x));
+  }
+};
+
+template <typename OutT>
+__device__ __forceinline__ void store4(OutT* p, const float (&v)[4]) {
+  uint2 w = make_uint2(Pack<OutT>::two(v[0], v[1]), Pack<OutT>::two(v[2], v[3]));
+  *reinterpret_cast<uint2*>(p) = w;
+}
+
+__device__ __forceinline__ void copy_rows(uint8_t* dst, const uint8_t* src, size_t bytes, int tid) {
+  const uint4* s = reinterpret_cast<const uint4*>(src);
+  uint4* d = reinterpret_cast<uint4*>(dst);
+  const size_t n = bytes / 16;
+  size_t i = tid;
+  for (; i + 3 * kThreads < n; i += 4 * kThreads) {
+    uint4 a = __ldcs(s + i), b = __ldcs(s + i + kThreads), c = __ldcs(s + i + 2 * kThreads),
+          e = __ldcs(s + i + 3 * kThreads);
+    d[i] = a;
+    d[i + kThreads] = b;
+    d[i + 2 * kThreads] = c;
+    d[i + 3 * kThreads] = e;
+  }
+  for (; i < n; i += kThreads) d[i] = __ldcs(s + i);
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(kThreads, 3)
+    assemble_kernel(const ChunkDesc* __restrict__ chunks, const float2* __restrict__ cs_table, ModelDims m,
+                    uint32_t* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t bars[kParts + 1];
+
+  const int tid = threadIdx.x;
+  const int item = blockIdx.x;
+  const int kv = item & 1;
+  const int l = (item >> 1) % m.L;
+  const int ci = (item >> 1) / m.L;
+  const ChunkDesc cd = chunks[ci];
+  const int H = m.Hkv, C = m.C;
+  constexpr int d = kHeadDim;
+  const size_t row_elems = (size_t)H * d;
+  const size_t dst_off = ((size_t)(l * 2 + kv) * cd.T + cd.new_pos) * row_elems;  // in elements
+  OutT* dst = reinterpret_cast<OutT*>(cd.kv_buf) + dst_off;
+  const size_t out_bytes = (size_t)C * row_elems * 2;
+
+  // ---- rows that are plain copies: FRESH chunks; unquantised values; unquantised keys that do not move
+  if (cd.mode == KVB_MODE_FRESH) {
+    copy_rows(reinterpret_cast<uint8_t*>(dst), cd.fresh + dst_off * 2, out_bytes, tid);
+    return;
+  }
+  if (cd.mode == KVB_MODE_FP16 && (kv == 1 || cd.delta_pos == 0)) {
+    copy_rows(reinterpret_cast<uint8_t*>(dst), (kv ? cd.v_src : cd.k_src) + (size_t)l * out_bytes, out_bytes, tid);
+    return;
+  }
+
+  // ---- staged path
+  const int bits = cd.mode == KVB_MODE_INT8 ? 8 : (cd.mode == KVB_MODE_INT4 ? 4 : 16);
+  const uint32_t code_bytes = (uint32_t)(C * row_elems * bits / 8);
+  const uint8_t* codes_g = (kv ? cd.v_src : cd.k_src) + (size_t)l * code_bytes;
+  uint32_t meta_bytes = 0;
+  const uint8_t* meta_g = nullptr;
+  int G = 1;  // key token groups, or value channel groups
+  if (bits != 16) {
+    if (!kv) {
+      G = bits == 8 ? 1 : C / m.int4_group;
+      meta_bytes = (uint32_t)(G * row_elems * 8);
+      meta_g = reinterpret_cast<const uint8_t*>(cd.k_meta) + (size_t)l * meta_bytes;
+    } else {
+      G = bits == 8 ? 1 : d / m.int4_group;
+      meta_bytes = (uint32_t)(C * H * G * 8);
+      meta_g = reinterpret_cast<const uint8_t*>(cd.v_meta) + (size_t)l * meta_bytes;
+    }
+  }
+  uint8_t* s_codes = smem;
+  const float* s_meta = reinterpret_cast<const float*>(smem + code_bytes);
+  const uint32_t part_bytes = code_bytes / kParts;
+
+  if (tid == 0) {
+    for (int i = 0; i <= kParts; ++i) mbar_init(&bars[i], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (tid == 0) {
+    if (meta_bytes) {
+      mbar_expect_tx(&bars[0], meta_bytes);
+      bulk_g2s(smem + code_bytes, meta_g, meta_bytes, &bars[0]);
+    }
+    for (int p = 0; p < kParts; ++p) {
+      mbar_expect_tx(&bars[1 + p], part_bytes);
+      bulk_g2s(s_codes + (size_t)p * part_bytes, codes_g + (size_t)p * part_bytes, part_bytes, &bars[1 + p]);
+    }
+  }
+
+  const int lane = tid & 31, warp = tid >> 5;
+  const int s = lane >> 4, ln = lane & 15;
+  const int hw = warp * 2 + s;  // half-warp 0..15
+  const int h = hw % H;
+  const int n_slots = 16 / H;
+  const int tok_per = C / n_slots;
+  const int t0 = (hw / H) * tok_per;
+  const int tok_per_part = C / kParts;
+  const int off_a = s ? 64 : 0, off_b = s ? 0 : 64;  // second half-warp reads the high half first (bank spread)
+  bool ok = true;
+  if (meta_bytes) ok = mbar_wait(&bars[0], 0);
+  int ready_part = -1;
+
+  if (!kv) {
+    // ------------------------------ keys
+    float A_lo[4], B_lo[4], C_lo[4], A_hi[4], B_hi[4], C_hi[4];
+    float cs_c[4], cs_s[4];
+    {
+      const float4* p = reinterpret_cast<const float4*>(cs_table + (size_t)ci * (d / 2) + 4 * ln);
+      float4 a = __ldg(p), b = __ldg(p + 1);
+      cs_c[0] = a.x, cs_s[0] = a.y, cs_c[1] = a.z, cs_s[1] = a.w;
+      cs_c[2] = b.x, cs_s[2] = b.y, cs_c[3] = b.z, cs_s[3] = b.w;
+    }
+    int cur_group = -1;
+    const int group_tokens = bits == 8 ? C : m.int4_group;
+#pragma unroll 2
+    for (int tt = 0; tt < tok_per; ++tt) {
+      const int t = t0 + tt;
+      const int part = t / tok_per_part;
+      if (part != ready_part) {
+        ok = ok && mbar_wait(&bars[1 + part], 0);
+        ready_part = part;
+      }
+      if (!ok) break;
+      const int u = t * H + h;
+      OutT* orow = dst + (size_t)u * d;
+      float ql[4], qh[4];
+      if (bits == 16) {
+        const uint8_t* row = s_codes + (size_t)u * (d * 2);
+        uint2 a = *reinterpret_cast<const uint2*>(row + 8 * ln);
+        uint2 b = *reinterpret_cast<const uint2*>(row + 128 + 8 * ln);
+        float2 f;
+        f = Pack<OutT>::unpack(a.x), ql[0] = f.x, ql[1] = f.y;
+        f = Pack<OutT>::unpack(a.y), ql[2] = f.x, ql[3] = f.y;
+        f = Pack<OutT>::unpack(b.x), qh[0] = f.x, qh[1] = f.y;
+        f = Pack<OutT>::unpack(b.y), qh[2] = f.x, qh[3] = f.y;
+        float ol[4], oh[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          ol[i] = fmaf(ql[i], cs_c[i], -(qh[i] * cs_s[i]));
+          oh[i] = fmaf(qh[i], cs_c[i], ql[i] * cs_s[i]);
+        }
+        store4(orow + 4 * ln, ol);
+        store4(orow + 64 + 4 * ln, oh);
+        continue;
+      }
+      const int g = t / group_tokens;
+      if (g != cur_group) {
+        cur_group = g;
+        const float* mlo = s_meta + ((size_t)(g * H + h) * d + 4 * ln) * 2;
+        const float4 a0 = *reinterpret_cast<const float4*>(mlo), a1 = *reinterpret_cast<const float4*>(mlo + 4);
+        const float4 b0 = *reinterpret_cast<const float4*>(mlo + 128), b1 = *reinterpret_cast<const float4*>(mlo + 132);
+        const float sl[4] = {a0.x, a0.z, a1.x, a1.z}, ml[4] = {a0.y, a0.w, a1.y, a1.w};
+        const float sh[4] = {b0.x, b0.z, b1.x, b1.z}, mh[4] = {b0.y, b0.w, b1.y, b1.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          A_lo[i] = sl[i] * cs_c[i];
+          B_lo[i] = -(sh[i] * cs_s[i]);
+          C_lo[i] = fmaf(ml[i], cs_c[i], -(mh[i] * cs_s[i]));
+          A_hi[i] = sh[i] * cs_c[i];
+          B_hi[i] = sl[i] * cs_s[i];
+          C_hi[i] = fmaf(mh[i], cs_c[i], ml[i] * cs_s[i]);
+        }
+      }
+      if (bits == 8) {
+        const uint8_t* row = s_codes + (size_t)u * d;
+        const uint32_t xa = *reinterpret_cast<const uint32_t*>(row + off_a + 4 * ln);
+        const uint32_t xb = *reinterpret_cast<const uint32_t*>(row + off_b + 4 * ln);
+        const uint32_t xl = s ? xb : xa, xh = s ? xa : xb;
+        ql[0] = byte_to_float<0>(xl), ql[1] = byte_to_float<1>(xl), ql[2] = byte_to_float<2>(xl), ql[3] = byte_to_float<3>(xl);
+        qh[0] = byte_to_float<0>(xh), qh[1] = byte_to_float<1>(xh), qh[2] = byte_to_float<2>(xh), qh[3] = byte_to_float<3>(xh);
+      } else {
+        const uint8_t* row = s_codes + (size_t)u * (d / 2);
+        const uint32_t xl = *reinterpret_cast<const uint16_t*>(row + 2 * ln);
+        const uint32_t xh = *reinterpret_cast<const uint16_t*>(row + 32 + 2 * ln);
+        ql[0] = nibble_to_float<0>(xl), ql[1] = nibble_to_float<1>(xl), ql[2] = nibble_to_float<2>(xl), ql[3] = nibble_to_float<3>(xl);
+        qh[0] = nibble_to_float<0>(xh), qh[1] = nibble_to_float<1>(xh), qh[2] = nibble_to_float<2>(xh), qh[3] = nibble_to_float<3>(xh);
+      }
+      float ol[4], oh[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        ol[i] = fmaf(A_lo[i], ql[i], fmaf(B_lo[i], qh[i], C_lo[i]));
+        oh[i] = fmaf(A_hi[i], qh[i], fmaf(B_hi[i], ql[i], C_hi[i]));
+      }
+      store4(orow + 4 * ln, ol);
+      store4(orow + 64 + 4 * ln, oh);
+    }
+  } else {
+    // ------------------------------ values (INT8 / INT4 only; never rotated)
+#pragma unroll 2
+    for (int tt = 0; tt < tok_per; ++tt) {
+      const int t = t0 + tt;
+      const int part = t / tok_per_part;
+      if (part != ready_part) {
+        ok = ok && mbar_wait(&bars[1 + part], 0);
+        ready_part = part;
+      }
+      if (!ok) break;
+      const int u = t * H + h;
+      OutT* orow = dst + (size_t)u * d;
+      float ql[4], qh[4];
+      float s_lo, m_lo, s_hi, m_hi;
+      if (bits == 8) {
+        const float2 sm = *reinterpret_cast<const float2*>(s_meta + (size_t)u * 2);
+        s_lo = s_hi = sm.x, m_lo = m_hi = sm.y;
+        const uint8_t* row = s_codes + (size_t)u * d;
+        const uint32_t xa = *reinterpret_cast<const uint32_t*>(row + off_a + 4 * ln);
+        const uint32_t xb = *reinterpret_cast<const uint32_t*>(row + off_b + 4 * ln);
+        const uint32_t xl = s ? xb : xa, xh = s ? xa : xb;
+        ql[0] = byte_to_float<0>(xl), ql[1] = byte_to_float<1>(xl), ql[2] = byte_to_float<2>(xl), ql[3] = byte_to_float<3>(xl);
+        qh[0] = byte_to_float<0>(xh), qh[1] = byte_to_float<1>(xh), qh[2] = byte_to_float<2>(xh), qh[3] = byte_to_float<3>(xh);
+      } else {
+        const int g_lo = (4 * ln) / m.int4_group, g_hi = (64 + 4 * ln) / m.int4_group;
+        const float2 a = *reinterpret_cast<const float2*>(s_meta + ((size_t)u * G + g_lo) * 2);
+        const float2 b = *reinterpret_cast<const float2*>(s_meta + ((size_t)u * G + g_hi) * 2);
+        s_lo = a.x, m_lo = a.y, s_hi = b.x, m_hi = b.y;
+        const uint8_t* row = s_codes + (size_t)u * (d / 2);
+        const uint32_t xl = *reinterpret_cast<const uint16_t*>(row + 2 * ln);
+        const uint32_t xh = *reinterpret_cast<const uint16_t*>(row + 32 + 2 * ln);
+        ql[0] = nibble_to_float<0>(xl), ql[1] = nibble_to_float<1>(xl), ql[2] = nibble_to_float<2>(xl), ql[3] = nibble_to_float<3>(xl);
+        qh[0] = nibble_to_float<0>(xh), qh[1] = nibble_to_float<1>(xh), qh[2] = nibble_to_float<2>(xh), qh[3] = nibble_to_float<3>(xh);
+      }
+      float ol[4], oh[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        ol[i] = fmaf(ql[i], s_lo, m_lo);
+        oh[i] = fmaf(qh[i], s_hi, m_hi);
+      }
+      store4(orow + 4 * ln, ol);
+      store4(orow + 64 + 4 * ln, oh);
+    }
+  }
+
+  if (!ok) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
+  // Every thread drains every barrier before the CTA may retire, so no bulk copy can still be
+  // writing this CTA's shared memory when it is handed to the next CTA.
+  bool all = true;
+  if (meta_bytes) all = mbar_wait(&bars[0], 0) && all;
+  for (int p = 0; p < kParts; ++p) all = mbar_wait(&bars[1 + p], 0) && all;
+  if (!all) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
+}
+
+// cos/sin of delta_pos * theta^(-2j/d) in double, stored as float (one thread per plane j)
+__global__ void rope_table_kernel(const ChunkDesc* __restrict__ chunks, int n_chunks, const double* __restrict__ inv_freq,
+                                  int half_d, float2* __restrict__ cs_table) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_chunks * half_d) return;
+  const int ci = i / half_d, j = i % half_d;
+  const double a = (double)chunks[ci].delta_pos * inv_freq[j];
+  double sn, c;
+  sincos(a, &sn, &c);
+  cs_table[i] = make_float2((float)c, (float)sn);
+}
+
+}  // namespace
+
+size_t assemble_smem_bytes(const ModelDims& m, int mode) {
+  const size_t E = (size_t)m.Hkv * m.d;
+  switch (mode) {
+    case KVB_MODE_FP16:
+      return (size_t)m.C * E * 2;
+    case KVB_MODE_INT8:
+      return (size_t)m.C * E + max(E * 8, (size_t)m.C * m.Hkv * 8);
+    case KVB_MODE_INT4:
+      return (size_t)m.C * E / 2 +
+             max((size_t)(m.C / m.int4_group) * E * 8, (size_t)m.C * m.Hkv * (m.d / m.int4_group) * 8);
+    default:
+      return 0;
+  }
+}
+
+cudaError_t assemble_configure(size_t max_smem) {
+  cudaError_t e = cudaFuncSetAttribute(assemble_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)max_smem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(assemble_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+}
+
+cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const double* inv_freq, int half_d,
+                              float2* cs_table, cudaStream_t st) {
+  const int n = n_chunks * half_d;
+  rope_table_kernel<<<(n + 127) / 128, 128, 0, st>>>(chunks, n_chunks, inv_freq, half_d, cs_table);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
+                            size_t smem_bytes, uint32_t* status, cudaStream_t st) {
+  const unsigned grid = (unsigned)n_chunks * m.L * 2;
+  if (m.dtype == KVB_DT_BF16)
+    assemble_kernel<__nv_bfloat16><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status);
+  else
+    assemble_kernel<__half><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status);
+  return cudaGetLastError();
+}
+
+}  // namespace kvb

@@ -1,0 +1,437 @@
+// Host side of libkvb: context, table validation, descriptor packing, launches.
+// Nothing here computes on the data path; every step of the path runs in the kernels.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "kvb_internal.h"
+
+using namespace kvb;
+
+namespace {
+constexpr int kSlots = 4;  // pinned staging ring: a slot is reused only after its copy has completed
+}
+
+struct kvb_ctx {
+  int device = 0;
+  kvb_model_desc model{};
+  kvb_limits limits{};
+  ModelDims dims{};
+  // device memory
+  double* inv_freq = nullptr;            // [d/2]
+  float2* cs_table = nullptr;            // [max_chunks][d/2] cos/sin of the chunk's rotation
+  uint8_t* arena_dev = nullptr;          // descriptors of the current call
+  unsigned long long* acc = nullptr;     // [max_tokens] fixed-point deviation sums (kept zero between calls)
+  uint32_t* status_dev = nullptr;
+  // pinned staging ring
+  uint8_t* staging = nullptr;
+  cudaEvent_t slot_done[kSlots]{};
+  bool slot_used[kSlots]{};
+  int next_slot = 0;
+  size_t arena_bytes = 0;
+  bool acc_dirty = false;
+  cudaStream_t last_stream = nullptr;
+  int64_t launches = 0;
+  char err[512] = {0};
+};
+
+namespace {
+
+int fail(kvb_ctx* c, int code, const char* fmt, ...) {
+  if (c) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c->err, sizeof(c->err), fmt, ap);
+    va_end(ap);
+  }
+  return code;
+}
+
+int cuda_fail(kvb_ctx* c, cudaError_t e, const char* what) {
+  return fail(c, KVB_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define KVB_CUDA(ctx, call)                                     \
+  do {                                                          \
+    cudaError_t e_ = (call);                                    \
+    if (e_ != cudaSuccess) return cuda_fail(ctx, e_, #call);    \
+  } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Takes the next staging slot (waiting for its previous copy if needed).
+int take_slot(kvb_ctx* c, uint8_t** host) {
+  const int s = c->next_slot;
+  c->next_slot = (s + 1) % kSlots;
+  if (c->slot_used[s]) KVB_CUDA(c, cudaEventSynchronize(c->slot_done[s]));
+  *host = c->staging + (size_t)s * c->arena_bytes;
+  return -(s + 1);  // negative = success, encodes the slot
+}
+
+int upload(kvb_ctx* c, int slot, const uint8_t* host, size_t bytes, cudaStream_t st) {
+  KVB_CUDA(c, cudaMemcpyAsync(c->arena_dev, host, bytes, cudaMemcpyHostToDevice, st));
+  KVB_CUDA(c, cudaEventRecord(c->slot_done[slot], st));
+  c->slot_used[slot] = true;
+  return KVB_OK;
+}
+
+// Checks one request's table: chunks in prompt order tiling [0, T) exactly, enums and pointers sane.
+int check_request(kvb_ctx* c, const kvb_request& r, int ri, bool need_payload) {
+  const int C = c->model.chunk_tokens;
+  if (r.T <= 0 || r.n_chunks <= 0 || !r.chunks) return fail(c, KVB_ERR_INVALID_ARG, "request %d: empty or NULL chunk table", ri);
+  if (r.T % C != 0 || r.n_chunks != r.T / C)
+    return fail(c, KVB_ERR_BAD_TABLE, "request %d: T=%d is not n_chunks=%d x chunk_tokens=%d", ri, r.T, r.n_chunks, C);
+  if (!r.kv_buf || !r.fresh) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL kv_buf or fresh", ri);
+  if (!aligned16(r.kv_buf) || !aligned16(r.fresh))
+    return fail(c, KVB_ERR_BAD_TABLE, "request %d: kv_buf / fresh must be 16-byte aligned", ri);
+  for (int i = 0; i < r.n_chunks; ++i) {
+    const kvb_chunk& k = r.chunks[i];
+    if (k.n_tokens != C) return fail(c, KVB_ERR_BAD_TABLE, "request %d chunk %d: n_tokens=%d, expected %d", ri, i, k.n_tokens, C);
+    if (k.new_pos != i * C)
+      return fail(c, KVB_ERR_BAD_TABLE, "request %d chunk %d: new_pos=%d leaves a gap or overlap (expected %d)", ri, i, k.new_pos, i * C);
+    if (k.mode < KVB_MODE_FRESH || k.mode > KVB_MODE_INT4) return fail(c, KVB_ERR_INVALID_ARG, "request %d chunk %d: bad mode %d", ri, i, k.mode);
+    if (k.match < KVB_MATCH_MISS || k.match > KVB_MATCH_APPROX) return fail(c, KVB_ERR_INVALID_ARG, "request %d chunk %d: bad match %d", ri, i, k.match);
+    if (k.mode == KVB_MODE_FRESH) continue;
+    if (k.orig_pos < 0 || k.orig_pos >= (1 << 24) || k.new_pos >= (1 << 24))
+      return fail(c, KVB_ERR_BAD_TABLE, "request %d chunk %d: position out of range [0, 2^24)", ri, i);
+    if (k.match == KVB_MATCH_EXACT && k.orig_pos != k.new_pos)
+      return fail(c, KVB_ERR_BAD_TABLE, "request %d chunk %d: EXACT match must keep its position (%d -> %d)", ri, i, k.orig_pos, k.new_pos);
+    if (!need_payload) continue;
+    if (!k.k_codes || !k.v_codes) return fail(c, KVB_ERR_INVALID_ARG, "request %d chunk %d: NULL codes", ri, i);
+    if (!aligned16(k.k_codes) || !aligned16(k.v_codes)) return fail(c, KVB_ERR_BAD_TABLE, "request %d chunk %d: codes must be 16-byte aligned", ri, i);
+    if (k.mode != KVB_MODE_FP16) {
+      if (!k.k_meta || !k.v_meta) return fail(c, KVB_ERR_INVALID_ARG, "request %d chunk %d: NULL metadata", ri, i);
+      if (!aligned16(k.k_meta) || !aligned16(k.v_meta)) return fail(c, KVB_ERR_BAD_TABLE, "request %d chunk %d: metadata must be 16-byte aligned", ri, i);
+    }
+  }
+  return KVB_OK;
+}
+
+int check_batch(kvb_ctx* c, const kvb_request* reqs, int n_req, bool need_payload, int* chunks_total, int64_t* tokens_total) {
+  if (!c) return KVB_ERR_INVALID_ARG;
+  if (n_req < 0 || (n_req > 0 && !reqs)) return fail(c, KVB_ERR_INVALID_ARG, "bad request array");
+  if (n_req > c->limits.max_requests) return fail(c, KVB_ERR_WORKSPACE, "%d requests > max_requests=%d", n_req, c->limits.max_requests);
+  int ch = 0;
+  int64_t tk = 0;
+  for (int r = 0; r < n_req; ++r) {
+    const int st = check_request(c, reqs[r], r, need_payload);
+    if (st != KVB_OK) return st;
+    ch += reqs[r].n_chunks;
+    tk += reqs[r].T;
+  }
+  if (ch > c->limits.max_chunks_total) return fail(c, KVB_ERR_WORKSPACE, "%d chunks > max_chunks_total=%d", ch, c->limits.max_chunks_total);
+  if (tk > c->limits.max_tokens_total) return fail(c, KVB_ERR_WORKSPACE, "%lld tokens > max_tokens_total=%lld", (long long)tk, (long long)c->limits.max_tokens_total);
+  *chunks_total = ch;
+  *tokens_total = tk;
+  return KVB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* kvb_status_string(int s) {
+  switch (s) {
+    case KVB_OK: return "ok";
+    case KVB_ERR_INVALID_ARG: return "invalid argument";
+    case KVB_ERR_BAD_TABLE: return "bad chunk table";
+    case KVB_ERR_UNSUPPORTED: return "unsupported shape or size";
+    case KVB_ERR_WORKSPACE: return "call exceeds the context's limits";
+    case KVB_ERR_CUDA: return "CUDA error";
+    case KVB_ERR_DEVICE_STATUS: return "device-side status set";
+    case KVB_ERR_NO_DEVICE: return "no usable GPU";
+    default: return "unknown status";
+  }
+}
+
+int kvb_select_count(int T, double ratio) {
+  if (T <= 0 || !(ratio > 0.0)) return 0;
+  const double k = floor(ratio * (double)T);
+  return k >= (double)T ? T : (int)k;
+}
+
+int kvb_validate(const kvb_model_desc* model, const kvb_limits* limits, const kvb_request* reqs, int n_req,
+                 int need_payload, char* err, size_t err_len) {
+  if (!model || !limits) return KVB_ERR_INVALID_ARG;
+  kvb_ctx tmp;  // no device resources: only the fields the checks read
+  tmp.model = *model;
+  tmp.limits = *limits;
+  int ch = 0;
+  int64_t tk = 0;
+  const int st = check_batch(&tmp, reqs, n_req, need_payload != 0, &ch, &tk);
+  if (err && err_len) snprintf(err, err_len, "%s", tmp.err);
+  return st;
+}
+
+const char* kvb_last_error(kvb_ctx* c) { return c ? c->err : "NULL context"; }
+int64_t kvb_launch_count(kvb_ctx* c) { return c ? c->launches : 0; }
+
+int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb_limits* limits) {
+  if (!out || !model || !limits) return KVB_ERR_INVALID_ARG;
+  *out = nullptr;
+  const kvb_model_desc& m = *model;
+  if (m.L <= 0 || m.Hq <= 0 || m.Hkv <= 0 || m.Hq % m.Hkv != 0 || !(m.rope_theta > 1.0) ||
+      (m.kv_dtype != KVB_DT_F16 && m.kv_dtype != KVB_DT_BF16) || limits->max_requests <= 0 ||
+      limits->max_chunks_total <= 0 || limits->max_tokens_total <= 0)
+    return KVB_ERR_INVALID_ARG;
+  const int rep = m.Hq / m.Hkv;
+  const bool pow2_h = (m.Hkv & (m.Hkv - 1)) == 0 && m.Hkv <= 16;
+  const bool pow2_rep = (rep & (rep - 1)) == 0 && rep <= 16;
+  if (m.d != 128 || m.chunk_tokens != 128 || m.int4_group != 32 || !pow2_h || !pow2_rep) return KVB_ERR_UNSUPPORTED;
+
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return KVB_ERR_NO_DEVICE;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess || prop.major != 10) return KVB_ERR_NO_DEVICE;
+
+  kvb_ctx* c = new (std::nothrow) kvb_ctx();
+  if (!c) return KVB_ERR_CUDA;
+  c->device = device;
+  c->model = m;
+  c->limits = *limits;
+  c->dims = ModelDims{m.L, m.Hq, m.Hkv, m.d, m.chunk_tokens, m.kv_dtype, m.int4_group};
+  *out = c;  // handed out even on failure so the caller can read the error text and destroy it
+
+  KVB_CUDA(c, cudaSetDevice(device));
+  size_t smem_max = 0;
+  for (int mode = KVB_MODE_FP16; mode <= KVB_MODE_INT4; ++mode) {
+    const size_t s = assemble_smem_bytes(c->dims, mode);
+    if (s > smem_max) smem_max = s;
+  }
+  if (smem_max > 200 * 1024) return fail(c, KVB_ERR_UNSUPPORTED, "chunk-layer block of %zu bytes does not fit shared memory", smem_max);
+  KVB_CUDA(c, assemble_configure(smem_max));
+  KVB_CUDA(c, topk_configure());
+  KVB_CUDA(c, attention_mma_configure());
+
+  const int half = m.d / 2;
+  std::vector<double> inv(half);
+  for (int j = 0; j < half; ++j) inv[j] = pow(m.rope_theta, -2.0 * (double)j / (double)m.d);
+  KVB_CUDA(c, cudaMalloc(&c->inv_freq, half * sizeof(double)));
+  KVB_CUDA(c, cudaMemcpy(c->inv_freq, inv.data(), half * sizeof(double), cudaMemcpyHostToDevice));
+  KVB_CUDA(c, cudaMalloc(&c->cs_table, (size_t)limits->max_chunks_total * half * sizeof(float2)));
+
+  const size_t a1 = sizeof(ChunkDesc) * (size_t)limits->max_chunks_total;
+  const size_t a2 = sizeof(ReqDesc) * (size_t)limits->max_requests + sizeof(SeamWindow) * (size_t)limits->max_chunks_total;
+  c->arena_bytes = ((a1 > a2 ? a1 : a2) + 255) & ~(size_t)255;
+  KVB_CUDA(c, cudaMalloc(&c->arena_dev, c->arena_bytes));
+  KVB_CUDA(c, cudaMallocHost(&c->staging, c->arena_bytes * kSlots));
+  for (int s = 0; s < kSlots; ++s) KVB_CUDA(c, cudaEventCreateWithFlags(&c->slot_done[s], cudaEventDisableTiming));
+  KVB_CUDA(c, cudaMalloc(&c->acc, (size_t)limits->max_tokens_total * sizeof(unsigned long long)));
+  KVB_CUDA(c, cudaMemset(c->acc, 0, (size_t)limits->max_tokens_total * sizeof(unsigned long long)));
+  KVB_CUDA(c, cudaMalloc(&c->status_dev, sizeof(uint32_t)));
+  KVB_CUDA(c, cudaMemset(c->status_dev, 0, sizeof(uint32_t)));
+  KVB_CUDA(c, cudaDeviceSynchronize());
+  return KVB_OK;
+}
+
+int kvb_destroy(kvb_ctx* c) {
+  if (!c) return KVB_ERR_INVALID_ARG;
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  cudaFree(c->inv_freq);
+  cudaFree(c->cs_table);
+  cudaFree(c->arena_dev);
+  cudaFree(c->acc);
+  cudaFree(c->status_dev);
+  if (c->staging) cudaFreeHost(c->staging);
+  for (int s = 0; s < kSlots; ++s)
+    if (c->slot_done[s]) cudaEventDestroy(c->slot_done[s]);
+  delete c;
+  return KVB_OK;
+}
+
+int kvb_last_status(kvb_ctx* c) {
+  if (!c) return KVB_ERR_INVALID_ARG;
+  KVB_CUDA(c, cudaSetDevice(c->device));
+  KVB_CUDA(c, cudaStreamSynchronize(c->last_stream));
+  uint32_t st = 0;
+  KVB_CUDA(c, cudaMemcpy(&st, c->status_dev, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st) return fail(c, KVB_ERR_DEVICE_STATUS, "device status word 0x%x", st);
+  return KVB_OK;
+}
+
+int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, true, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  ChunkDesc* cd = reinterpret_cast<ChunkDesc*>(host);
+  size_t smem = 0;
+  int n = 0;
+  for (int r = 0; r < n_req; ++r) {
+    for (int i = 0; i < reqs[r].n_chunks; ++i, ++n) {
+      const kvb_chunk& k = reqs[r].chunks[i];
+      ChunkDesc d{};
+      d.k_src = static_cast<const uint8_t*>(k.k_codes);
+      d.v_src = static_cast<const uint8_t*>(k.v_codes);
+      d.k_meta = static_cast<const float*>(k.k_meta);
+      d.v_meta = static_cast<const float*>(k.v_meta);
+      d.kv_buf = static_cast<uint8_t*>(reqs[r].kv_buf);
+      d.fresh = static_cast<const uint8_t*>(reqs[r].fresh);
+      d.T = reqs[r].T;
+      d.new_pos = k.new_pos;
+      d.delta_pos = k.mode == KVB_MODE_FRESH ? 0 : k.new_pos - k.orig_pos;
+      d.mode = k.mode;
+      cd[n] = d;
+      const size_t s = assemble_smem_bytes(c->dims, k.mode);
+      if (s > smem) smem = s;
+    }
+  }
+  const int up = upload(c, slot, host, sizeof(ChunkDesc) * (size_t)n, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  const ChunkDesc* cd_dev = reinterpret_cast<const ChunkDesc*>(c->arena_dev);
+  KVB_CUDA(c, launch_rope_table(cd_dev, n, c->inv_freq, c->model.d / 2, c->cs_table, st));
+  KVB_CUDA(c, launch_assemble(cd_dev, n, c->cs_table, c->dims, smem, c->status_dev, st));
+  c->launches += 2;
+  return KVB_OK;
+}
+
+int kvb_deviation_topk(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_select_params* p,
+                       const kvb_selection* out, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  if (!p || !out) return fail(c, KVB_ERR_INVALID_ARG, "NULL select params or outputs");
+  if ((p->which & 3) == 0 || (p->which & ~3) || p->seam_before < 0 || p->seam_after < 0 ||
+      (p->k_override < 0 && !(p->ratio >= 0.0 && p->ratio <= 1.0)))
+    return fail(c, KVB_ERR_INVALID_ARG, "bad select params");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
+  SeamWindow* sw = reinterpret_cast<SeamWindow*>(host + sizeof(ReqDesc) * (size_t)n_req);
+  const int tile_tok = deviation_tile_tokens();
+  int tiles = 0, tok = 0, n_seams = 0, max_T = 0, max_k = 0;
+  for (int r = 0; r < n_req; ++r) {
+    const kvb_request& q = reqs[r];
+    const kvb_selection& o = out[r];
+    if (!o.delta || !o.rank || !o.sel || !o.n_sel) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL selection output", r);
+    const int k = p->k_override >= 0 ? p->k_override : kvb_select_count(q.T, p->ratio);
+    if (k > q.T) return fail(c, KVB_ERR_INVALID_ARG, "request %d: k=%d > T=%d", r, k, q.T);
+    if (q.T > topk_max_T() || k > topk_max_k())
+      return fail(c, KVB_ERR_UNSUPPORTED, "request %d: T=%d or k=%d beyond the selection kernel's limits (%d, %d)", r, q.T, k, topk_max_T(), topk_max_k());
+    if (o.sel_capacity < k) return fail(c, KVB_ERR_INVALID_ARG, "request %d: sel_capacity=%d < k=%d", r, o.sel_capacity, k);
+    ReqDesc d{};
+    d.kv_buf = static_cast<const uint8_t*>(q.kv_buf);
+    d.fresh = static_cast<const uint8_t*>(q.fresh);
+    d.delta = o.delta;
+    d.rank = o.rank;
+    d.sel = o.sel;
+    d.n_sel = o.n_sel;
+    d.T = q.T;
+    d.k = k;
+    d.sel_capacity = o.sel_capacity;
+    d.tok_offset = tok;
+    d.tile_offset = tiles;
+    d.seam_offset = n_seams;
+    // seams: interior boundaries with a cached chunk on either side (Algorithm 1 works on cached chunks)
+    for (int i = 1; i < q.n_chunks; ++i) {
+      if (q.chunks[i].mode == KVB_MODE_FRESH && q.chunks[i - 1].mode == KVB_MODE_FRESH) continue;
+      if (p->seam_before == 0 && p->seam_after == 0) continue;
+      const int pos = q.chunks[i].new_pos;
+      SeamWindow w;
+      w.lo = pos - p->seam_before < 0 ? 0 : pos - p->seam_before;
+      w.hi = pos + p->seam_after > q.T ? q.T : pos + p->seam_after;
+      sw[n_seams++] = w;
+    }
+    d.n_seams = n_seams - d.seam_offset;
+    rd[r] = d;
+    tok += q.T;
+    tiles += (q.T + tile_tok - 1) / tile_tok;
+    if (q.T > max_T) max_T = q.T;
+    if (k > max_k) max_k = k;
+  }
+  if (c->acc_dirty) {
+    KVB_CUDA(c, cudaMemsetAsync(c->acc, 0, (size_t)c->limits.max_tokens_total * sizeof(unsigned long long), st));
+    c->acc_dirty = false;
+  }
+  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req + sizeof(SeamWindow) * (size_t)n_seams, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  const ReqDesc* rd_dev = reinterpret_cast<const ReqDesc*>(c->arena_dev);
+  const SeamWindow* sw_dev = reinterpret_cast<const SeamWindow*>(c->arena_dev + sizeof(ReqDesc) * (size_t)n_req);
+  c->acc_dirty = true;  // cleared again once both kernels are in the stream
+  KVB_CUDA(c, launch_deviation(rd_dev, n_req, tiles, c->dims, p->which, c->acc, st));
+  const int n_terms = c->model.L * c->model.Hkv * ((p->which & 1) + ((p->which >> 1) & 1));
+  KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_terms, max_T, max_k, c->acc, c->status_dev, st));
+  c->acc_dirty = false;
+  c->launches += 2;
+  return KVB_OK;
+}
+
+int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_selection* sel, const void* const* q,
+                       void* const* out, float softmax_scale, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  if (!sel || !q || !out) return fail(c, KVB_ERR_INVALID_ARG, "NULL selection, q or out array");
+  if (!(softmax_scale > 0.f)) return fail(c, KVB_ERR_INVALID_ARG, "softmax_scale must be positive");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
+  const int tok_per_tile = 128 / (c->model.Hq / c->model.Hkv);
+  int tiles = 0;
+  for (int r = 0; r < n_req; ++r) {
+    const kvb_selection& s = sel[r];
+    if (!s.sel || !s.n_sel || s.sel_capacity <= 0 || !q[r] || !out[r])
+      return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL sel / n_sel / q / out or empty capacity", r);
+    if (!aligned16(q[r]) || !aligned16(out[r])) return fail(c, KVB_ERR_BAD_TABLE, "request %d: q / out must be 16-byte aligned", r);
+    ReqDesc d{};
+    d.kv_buf = static_cast<const uint8_t*>(reqs[r].kv_buf);
+    d.sel = s.sel;
+    d.n_sel = s.n_sel;
+    d.q = static_cast<const uint8_t*>(q[r]);
+    d.out = static_cast<uint8_t*>(out[r]);
+    d.T = reqs[r].T;
+    d.sel_capacity = s.sel_capacity;
+    d.tile_offset = tiles;
+    rd[r] = d;
+    tiles += (s.sel_capacity + tok_per_tile - 1) / tok_per_tile;
+  }
+  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  KVB_CUDA(c, launch_attention_mma(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, tiles, c->dims, softmax_scale, st));
+  c->launches += 1;
+  return KVB_OK;
+}
+
+int kvb_quantize_chunk(kvb_ctx* c, const void* x, int is_value, int bits, void* codes, void* meta, void* cuda_stream) {
+  if (!c) return KVB_ERR_INVALID_ARG;
+  if (!x || !codes || !meta || (bits != 4 && bits != 8)) return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(meta)) return fail(c, KVB_ERR_BAD_TABLE, "quantize buffers must be 16-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+  c->last_stream = st;
+  KVB_CUDA(c, launch_quantize(x, is_value ? 1 : 0, bits, codes, meta, c->dims, st));
+  c->launches += 1;
+  return KVB_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+// Internal declarations shared by the host side of libkvb and its kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvb.h"
+
+namespace kvb {
+
+// Sticky device status bits (ORed into the context's status word by kernels).
+enum : uint32_t {
+  DEV_STATUS_WAIT_TIMEOUT = 1u << 0,  // a bounded mbarrier wait gave up
+  DEV_STATUS_BAD_DESC = 1u << 1,      // a descriptor failed a device-side range check
+  DEV_STATUS_SEL_OVERFLOW = 1u << 2,  // selection did not fit sel_capacity
+};
+
+// One chunk of one request, as the assemble kernel sees it (device memory).
+struct ChunkDesc {
+  const uint8_t* k_src;  // codes of all layers; unused for FRESH
+  const uint8_t* v_src;
+  const float* k_meta;
+  const float* v_meta;
+  uint8_t* kv_buf;       // request's [L][2][T][H][d] buffer
+  const uint8_t* fresh;  // request's fresh tensor
+  int32_t T;
+  int32_t new_pos;
+  int32_t delta_pos;     // new_pos - orig_pos
+  int32_t mode;
+};
+
+// One request, as the deviation / top-k / attention kernels see it.
+struct ReqDesc {
+  const uint8_t* kv_buf;
+  const uint8_t* fresh;
+  float* delta;
+  int32_t* rank;
+  int32_t* sel;
+  int32_t* n_sel;
+  const uint8_t* q;
+  uint8_t* out;
+  int32_t T;
+  int32_t k;             // number of top-k entries
+  int32_t sel_capacity;
+  int32_t tok_offset;    // first token of this request in the call's flat token space
+  int32_t tile_offset;   // first tile of this request in a kernel's flat tile space
+  int32_t seam_offset;   // first entry of this request in the seam window list
+  int32_t n_seams;
+  int32_t pad;
+};
+
+struct SeamWindow {
+  int32_t lo, hi;  // [lo, hi)
+};
+
+struct ModelDims {
+  int L, Hq, Hkv, d, C, dtype, int4_group;
+};
+
+// ---- launchers (each defined next to its kernel) ----
+cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const double* inv_freq, int half_d,
+                              float2* cs_table, cudaStream_t st);
+cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
+                            size_t smem_bytes, uint32_t* status, cudaStream_t st);
+size_t assemble_smem_bytes(const ModelDims& m, int mode);
+cudaError_t assemble_configure(size_t max_smem);
+
+cudaError_t launch_deviation(const ReqDesc* reqs, int n_req, int total_tiles, const ModelDims& m, int which,
+                             unsigned long long* acc, cudaStream_t st);
+int deviation_tile_tokens();
+
+cudaError_t launch_topk(const ReqDesc* reqs, int n_req, const SeamWindow* seams, const ModelDims& m, int n_terms,
+                        int max_T, int max_k, unsigned long long* acc, uint32_t* status, cudaStream_t st);
+cudaError_t topk_configure();
+int topk_max_T();
+int topk_max_k();
+
+cudaError_t launch_attention_mma(const ReqDesc* reqs, int n_req, int total_tiles, const ModelDims& m, float scale,
+                                 cudaStream_t st);
+cudaError_t attention_mma_configure();
+
+cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
+                            cudaStream_t st);
+
+}  // namespace kvb
