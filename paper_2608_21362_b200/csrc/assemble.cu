@@ -24,6 +24,10 @@ constexpr int kParts = 4;
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr int kHeadDim = 128;
 
+// CTAs per (chunk, layer, K|V): 1 for up to 2 KV heads, H/2 beyond, so a CTA never stages more
+// than 256 (token, head) rows.
+__host__ __device__ inline int assemble_split(int H) { return H > 2 ? H / 2 : 1; }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -119,17 +123,23 @@ __global__ void __launch_bounds__(kThreads, 3)
   __shared__ __align__(8) uint64_t bars[kParts + 1];
 
   const int tid = threadIdx.x;
-  const int item = blockIdx.x;
+  const int H = m.Hkv;
+  const int split = assemble_split(H);  // CTAs per chunk-layer, so that a CTA stages at most 256 rows
+  int item = blockIdx.x;
+  const int part_id = item % split;
+  item /= split;
   const int kv = item & 1;
   const int l = (item >> 1) % m.L;
   const int ci = (item >> 1) / m.L;
   const ChunkDesc cd = chunks[ci];
-  const int H = m.Hkv, C = m.C;
+  const int C = m.C / split;            // tokens of this CTA
+  const int tb = part_id * C;           // first token of this CTA within the chunk
   constexpr int d = kHeadDim;
   const size_t row_elems = (size_t)H * d;
-  const size_t dst_off = ((size_t)(l * 2 + kv) * cd.T + cd.new_pos) * row_elems;  // in elements
+  const size_t dst_off = ((size_t)(l * 2 + kv) * cd.T + cd.new_pos + tb) * row_elems;  // in elements
   OutT* dst = reinterpret_cast<OutT*>(cd.kv_buf) + dst_off;
   const size_t out_bytes = (size_t)C * row_elems * 2;
+  const size_t layer_out_bytes = (size_t)m.C * row_elems * 2;
 
   // ---- rows that are plain copies: FRESH chunks; unquantised values; unquantised keys that do not move
   if (cd.mode == KVB_MODE_FRESH) {
@@ -137,26 +147,31 @@ __global__ void __launch_bounds__(kThreads, 3)
     return;
   }
   if (cd.mode == KVB_MODE_FP16 && (kv == 1 || cd.delta_pos == 0)) {
-    copy_rows(reinterpret_cast<uint8_t*>(dst), (kv ? cd.v_src : cd.k_src) + (size_t)l * out_bytes, out_bytes, tid);
+    copy_rows(reinterpret_cast<uint8_t*>(dst), (kv ? cd.v_src : cd.k_src) + (size_t)l * layer_out_bytes + (size_t)tb * row_elems * 2,
+              out_bytes, tid);
     return;
   }
 
   // ---- staged path
   const int bits = cd.mode == KVB_MODE_INT8 ? 8 : (cd.mode == KVB_MODE_INT4 ? 4 : 16);
-  const uint32_t code_bytes = (uint32_t)(C * row_elems * bits / 8);
-  const uint8_t* codes_g = (kv ? cd.v_src : cd.k_src) + (size_t)l * code_bytes;
+  const uint32_t code_bytes = (uint32_t)(C * row_elems * bits / 8);  // this CTA's share of the layer's codes
+  const uint8_t* codes_g = (kv ? cd.v_src : cd.k_src) + ((size_t)l * split + part_id) * code_bytes;
   uint32_t meta_bytes = 0;
   const uint8_t* meta_g = nullptr;
-  int G = 1;  // key token groups, or value channel groups
+  int G = 1;        // value channel groups per row
+  int g_first = 0;  // first key token group held in shared memory
+  const int group_tokens = bits == 8 ? m.C : m.int4_group;
   if (bits != 16) {
     if (!kv) {
-      G = bits == 8 ? 1 : C / m.int4_group;
-      meta_bytes = (uint32_t)(G * row_elems * 8);
-      meta_g = reinterpret_cast<const uint8_t*>(cd.k_meta) + (size_t)l * meta_bytes;
+      const int G_layer = m.C / group_tokens;
+      g_first = tb / group_tokens;
+      const int n_g = (tb + C - 1) / group_tokens - g_first + 1;
+      meta_bytes = (uint32_t)(n_g * row_elems * 8);
+      meta_g = reinterpret_cast<const uint8_t*>(cd.k_meta) + ((size_t)l * G_layer + g_first) * row_elems * 8;
     } else {
       G = bits == 8 ? 1 : d / m.int4_group;
       meta_bytes = (uint32_t)(C * H * G * 8);
-      meta_g = reinterpret_cast<const uint8_t*>(cd.v_meta) + (size_t)l * meta_bytes;
+      meta_g = reinterpret_cast<const uint8_t*>(cd.v_meta) + ((size_t)l * split + part_id) * meta_bytes;
     }
   }
   uint8_t* s_codes = smem;
@@ -203,7 +218,6 @@ __global__ void __launch_bounds__(kThreads, 3)
       cs_c[2] = b.x, cs_s[2] = b.y, cs_c[3] = b.z, cs_s[3] = b.w;
     }
     int cur_group = -1;
-    const int group_tokens = bits == 8 ? C : m.int4_group;
 #pragma unroll 2
     for (int tt = 0; tt < tok_per; ++tt) {
       const int t = t0 + tt;
@@ -235,7 +249,7 @@ __global__ void __launch_bounds__(kThreads, 3)
         store4(orow + 64 + 4 * ln, oh);
         continue;
       }
-      const int g = t / group_tokens;
+      const int g = (tb + t) / group_tokens - g_first;
       if (g != cur_group) {
         cur_group = g;
         const float* mlo = s_meta + ((size_t)(g * H + h) * d + 4 * ln) * 2;
@@ -347,14 +361,15 @@ __global__ void rope_table_kernel(const ChunkDesc* __restrict__ chunks, int n_ch
 
 size_t assemble_smem_bytes(const ModelDims& m, int mode) {
   const size_t E = (size_t)m.Hkv * m.d;
+  const size_t C = (size_t)m.C / assemble_split(m.Hkv);  // tokens per CTA
+  auto mx = [](size_t a, size_t b) { return a > b ? a : b; };
   switch (mode) {
     case KVB_MODE_FP16:
-      return (size_t)m.C * E * 2;
+      return C * E * 2;
     case KVB_MODE_INT8:
-      return (size_t)m.C * E + max(E * 8, (size_t)m.C * m.Hkv * 8);
+      return C * E + mx(E * 8, C * m.Hkv * 8);
     case KVB_MODE_INT4:
-      return (size_t)m.C * E / 2 +
-             max((size_t)(m.C / m.int4_group) * E * 8, (size_t)m.C * m.Hkv * (m.d / m.int4_group) * 8);
+      return C * E / 2 + mx(((C + m.int4_group - 1) / m.int4_group) * E * 8, C * m.Hkv * (m.d / m.int4_group) * 8);
     default:
       return 0;
   }
@@ -376,7 +391,7 @@ cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const doubl
 
 cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
                             size_t smem_bytes, uint32_t* status, cudaStream_t st) {
-  const unsigned grid = (unsigned)n_chunks * m.L * 2;
+  const unsigned grid = (unsigned)n_chunks * m.L * 2 * assemble_split(m.Hkv);
   if (m.dtype == KVB_DT_BF16)
     assemble_kernel<__nv_bfloat16><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status);
   else
