@@ -168,6 +168,26 @@ int kvb_selective_attn(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const k
 int kvb_quantize_chunk(kvb_ctx* ctx, const void* x, int is_value, int bits, void* codes, void* meta,
                        void* cuda_stream);
 
+/* Cosine deviation of ONE request for callers that cannot allocate GPU memory:
+ * a server that gave the whole GPU to its own block pool at start-up, or a
+ * latency-critical thread that may not take the device-wide synchronisation an
+ * allocation implies.  (The paper has no counterpart; the arithmetic is that of
+ * kvb_deviation_topk's deviation step, Algorithm 2 step 2.)  Needs no context
+ * and calls no cudaMalloc / cudaFree: its scratch (fixed-point sums and one
+ * descriptor) is a static device array of 128 KiB + 256 bytes that every GPU
+ * loading this library holds until the process exits.
+ *   kv_buf, fresh  device, [L][2][T][H][d] in model->kv_dtype, 16-byte aligned
+ *   delta          device, [T] float32, written
+ *   T              1 .. 16384; larger returns KVB_ERR_WORKSPACE (use a context)
+ *   which          bit 0 keys, bit 1 values
+ * Asynchronous on cuda_stream.  The first call on a device resolves the array's
+ * device address (cudaGetSymbolAddress) and should come before any stream
+ * capture.  All calls share the one array, which keeps the previous call's
+ * contents (this call clears what it sums into): two calls whose GPU work
+ * overlaps, e.g. on different streams, race on it. */
+int kvb_deviation_static(int device, const kvb_model_desc* model, const void* kv_buf, const void* fresh, int T,
+                         int which, float* delta, void* cuda_stream);
+
 /* Host-only: runs the table checks the data-path calls run before launching
  * (chunks in prompt order tiling [0,T), enums, positions, pointer alignment,
  * the limits) without touching a GPU.  need_payload != 0 also requires the

@@ -242,6 +242,15 @@ def kvb_quantize_chunk(ctx, x: torch.Tensor, is_value: bool, bits: int, codes: t
     return _check(ctx, st) if check else st
 
 
+def kvb_deviation_static(device: int, model: kvb_model_desc, kv_buf: torch.Tensor, fresh: torch.Tensor, T: int,
+                         which: int, delta: torch.Tensor, stream=None) -> int:
+    """Deviation of one request without a context and without any allocation (static device scratch,
+    T <= 16384).  Returns the status code; the caller owns kv_buf, fresh and delta."""
+    L = lib()
+    L.kvb_deviation_static.argtypes = [C.c_int, C.POINTER(kvb_model_desc), C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
+    return int(L.kvb_deviation_static(device, C.byref(model), kv_buf.data_ptr(), fresh.data_ptr(), T, which, delta.data_ptr(), _stream(stream)))
+
+
 def kvb_last_status(ctx, check: bool = True) -> int:
     st = lib().kvb_last_status(ctx)
     return _check(ctx, st) if check else st
