@@ -1,0 +1,477 @@
+// Selected-row causal attention (Eq. 2) on the 5th-generation tensor cores.
+//
+// One CTA per (layer, KV head, tile of selected tokens); a tile packs TOK = 128/rep selected
+// tokens times the rep = Hq/Hkv query heads sharing the KV head into the 128 rows of one
+// tcgen05.mma (M = 128).  Keys go by blocks of 128:
+//     S = Q K^T   tcgen05.mma, Q and K from shared memory (K-major, 128-byte swizzle), S in TMEM
+//     P = exp2(scale*S - m)  by 128 threads, one TMEM lane (row) each, written back over S as bf16
+//     O += P V    tcgen05.mma, P from TMEM, V from shared memory (MN-major), O in TMEM
+// Tiles are fetched by TMA (cp.async.bulk.tensor) with mbarrier completion.  Warp roles: warp 0
+// lane 0 issues TMA, warp 1 lane 0 issues MMAs (and owns the TMEM allocation), warps 2-5 do the
+// softmax and the epilogue.  Each CTA uses 256 TMEM columns and 96 KB of shared memory so that two
+// CTAs share an SM: one CTA's softmax overlaps the other's MMAs.
+//
+// The running maximum is lazy: the reference m only moves when a block's maximum exceeds it by
+// more than 8 (a factor 256), in which case the O rows in TMEM are rescaled; P stays within
+// [0, 256] otherwise, which costs nothing in bf16.
+// Every wait is bounded; a wait that runs out raises an abort flag, all roles fall through to the
+// common teardown (TMEM is released) and the context's status word records it.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "kvb_internal.h"
+
+namespace kvb {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kRows = 128;
+constexpr int kBlockKeys = 128;
+constexpr int kD = 128;
+constexpr uint32_t kTileBytes = kRows * kD * 2;      // 32 KB: Q, K or V tile
+constexpr uint32_t kHalfBytes = kTileBytes / 2;      // one 64-element-wide TMA box
+constexpr uint32_t kTmemCols = 256;                  // S/P: columns 0..127, O: columns 128..255
+constexpr uint32_t kWaitLimit = 1u << 24;
+constexpr float kLazyThreshold = 8.0f;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// ---- mbarrier
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  for (uint32_t i = 0; i < kWaitLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 255u) == 255u) {
+      if (*abort_flag) return false;
+      __nanosleep(128);
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+
+// ---- TMA
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(
+                   smem_u32(dst)),
+               "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(
+                   smem_u32(dst)),
+               "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+               : "memory");
+}
+__device__ __forceinline__ void tensormap_acquire(const CUtensorMap* map) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+// ---- tcgen05
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Load 32 columns of this thread's TMEM lane and wait for them: the wait sits in the same asm
+// statement so that no use of the registers can be scheduled before it.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]),
+      "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]),
+      "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
+      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (128-byte swizzle, 8-row groups 1024 bytes apart).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version of this architecture
+  d |= 2ull << 61;  // SWIZZLE_128B
+  return d;
+}
+
+// Instruction descriptor: float32 accumulate, A/B bf16 or fp16, M = 128, N = 128.
+template <int DT>
+__device__ __forceinline__ uint32_t instr_desc(bool b_mn_major) {
+  const uint32_t fmt = DT == KVB_DT_BF16 ? 1u : 0u;
+  uint32_t d = 0;
+  d |= 1u << 4;                      // D format f32
+  d |= fmt << 7;                     // A format
+  d |= fmt << 10;                    // B format
+  d |= (b_mn_major ? 1u : 0u) << 16; // B major: 0 = K, 1 = MN
+  d |= (128u >> 3) << 17;            // N
+  d |= (128u >> 4) << 24;            // M
+  return d;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int DT>
+__device__ __forceinline__ uint32_t pack2(float a, float b) {
+  if (DT == KVB_DT_BF16) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+  } else {
+    __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+  }
+}
+
+struct __align__(8) Barriers {
+  uint64_t q_full, k_full, k_empty, v_full, v_empty, s_full, p_full, o_full;
+};
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 2)
+    attn_tc_kernel(const ReqDesc* __restrict__ reqs, const CUtensorMap* __restrict__ maps, int n_req, int total_tiles,
+                   ModelDims m, float scale_log2, uint32_t* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Barriers bars;
+  __shared__ uint32_t s_tmem_base;
+  __shared__ uint32_t s_abort;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per_tile = m.Hkv * m.L;
+  const int lin = blockIdx.x;
+  const int tile_flat = total_tiles - 1 - lin / per_tile;  // longest tiles first
+  const int hk = (lin % per_tile) % m.Hkv;
+  const int l = (lin % per_tile) / m.Hkv;
+  int lo = 0, hi = n_req - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (reqs[mid].tile_offset <= tile_flat) lo = mid; else hi = mid - 1;
+  }
+  const ReqDesc rq = reqs[lo];
+  const CUtensorMap* map_q = maps + 2 * lo;
+  const CUtensorMap* map_kv = maps + 2 * lo + 1;
+  const int rep = m.Hq / m.Hkv;
+  const int TOK = kRows / rep;
+  const int tile = tile_flat - rq.tile_offset;
+  const int n_sel = min(*rq.n_sel, rq.sel_capacity);
+  const int i_base = tile * TOK;
+  if (i_base >= n_sel) return;  // uniform for the CTA, before anything is allocated
+  const int T = rq.T;
+  const int t_max = min(rq.sel[min(i_base + TOK, n_sel) - 1], T - 1);
+  const int nkb = t_max / kBlockKeys + 1;
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + kTileBytes;
+  uint8_t* sV = smem + 2 * kTileBytes;
+  volatile uint32_t* abort_flag = &s_abort;
+
+  if (tid == 0) {
+    mbar_init(&bars.q_full, 1);
+    mbar_init(&bars.k_full, 1);
+    mbar_init(&bars.k_empty, 1);
+    mbar_init(&bars.v_full, 1);
+    mbar_init(&bars.v_empty, 1);
+    mbar_init(&bars.s_full, 1);
+    mbar_init(&bars.p_full, 128);
+    mbar_init(&bars.o_full, 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM allocation is a warp-wide operation
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = s_tmem_base;
+  const uint32_t tmem_S = tmem_base;        // also P (packed 16-bit pairs, columns 0..63)
+  const uint32_t tmem_O = tmem_base + 128;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      tensormap_acquire(map_q);
+      tensormap_acquire(map_kv);
+      mbar_expect_tx(&bars.q_full, kTileBytes);
+      tma_load_4d(sQ, map_q, 0, hk * rep, i_base, l, &bars.q_full);
+      tma_load_4d(sQ + kHalfBytes, map_q, 64, hk * rep, i_base, l, &bars.q_full);
+      bool ok = true;
+      for (int j = 0; j < nkb && ok; ++j) {
+        if (j > 0) ok = mbar_wait(&bars.k_empty, (j - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(&bars.k_full, kTileBytes);
+        tma_load_5d(sK, map_kv, 0, hk, j * kBlockKeys, 0, l, &bars.k_full);
+        tma_load_5d(sK + kHalfBytes, map_kv, 64, hk, j * kBlockKeys, 0, l, &bars.k_full);
+        if (j > 0) ok = mbar_wait(&bars.v_empty, (j - 1) & 1, abort_flag);
+        if (!ok) break;
+        mbar_expect_tx(&bars.v_full, kTileBytes);
+        tma_load_5d(sV, map_kv, 0, hk, j * kBlockKeys, 1, l, &bars.v_full);
+        tma_load_5d(sV + kHalfBytes, map_kv, 64, hk, j * kBlockKeys, 1, l, &bars.v_full);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_s = instr_desc<DT>(false);
+      const uint32_t idesc_pv = instr_desc<DT>(true);
+      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+      bool ok = mbar_wait(&bars.q_full, 0, abort_flag);
+      for (int j = 0; j < nkb && ok; ++j) {
+        ok = mbar_wait(&bars.k_full, j & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {  // 16 elements of d per step; 4 steps per 64-element box
+          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+          mma_ss(tmem_S, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+        }
+        tc_commit(&bars.s_full);
+        tc_commit(&bars.k_empty);
+        ok = mbar_wait(&bars.p_full, j & 1, abort_flag) && mbar_wait(&bars.v_full, j & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {  // 16 keys per step = 2048 bytes of V; the two 64-wide halves of d are 16 KB apart
+          mma_ts(tmem_O, tmem_S + ks * 8, smem_desc(v_addr + ks * 2048, kHalfBytes, 1024), idesc_pv, (j > 0 || ks > 0));
+        }
+        tc_commit(&bars.v_empty);
+      }
+      if (ok) tc_commit(&bars.o_full);
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue (warps 2..5)
+    const int quarter = warp & 3;              // TMEM lanes this warp may touch
+    const int row = quarter * 32 + lane;       // row of the tile = TMEM lane
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const int i_row = i_base + row / rep;
+    const int t_row = i_row < n_sel ? rq.sel[i_row] : -1;
+    int warp_tmin = t_row;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) warp_tmin = min(warp_tmin, __shfl_xor_sync(0xffffffffu, warp_tmin, o));
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool ok = true;
+    for (int j = 0; j < nkb; ++j) {
+      ok = mbar_wait(&bars.s_full, j & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after();
+      const int key0 = j * kBlockKeys;
+      const bool need_mask = key0 + kBlockKeys - 1 > warp_tmin;
+      // pass 1: block maximum of this row
+      float bm = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_S + lane_addr + c * 32, r);
+        if (need_mask) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (key0 + c * 32 + i <= t_row) bm = fmaxf(bm, __uint_as_float(r[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) bm = fmaxf(bm, __uint_as_float(r[i]));
+        }
+      }
+      bm *= scale_log2;  // scale_log2 > 0, so the maximum commutes with the scaling
+      // lazy reference maximum; O rows are rescaled only when the reference moves
+      float factor = 1.f;
+      if (bm > m_ref + kLazyThreshold || m_ref == -INFINITY) {
+        if (bm > -INFINITY) {
+          factor = m_ref == -INFINITY ? 0.f : exp2f(m_ref - bm);
+          m_ref = bm;
+        }
+      }
+      const bool rescale = j > 0 && __any_sync(0xffffffffu, factor != 1.f);
+      if (rescale) {  // PV of the previous block is complete: S of this block was issued after it
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t r[32];
+          tmem_ld32(tmem_O + lane_addr + c * 32, r);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * factor);
+          tmem_st32(tmem_O + lane_addr + c * 32, r);
+        }
+      }
+      l_sum *= factor;
+      const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+      // pass 2: P = exp2(scale*S - m), packed to 16 bits over the S columns already consumed
+      float psum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_S + lane_addr + c * 32, r);
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 32; i += 2) {
+          float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_use));
+          float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_use));
+          if (need_mask) {
+            if (key0 + c * 32 + i > t_row) p0 = 0.f;
+            if (key0 + c * 32 + i + 1 > t_row) p1 = 0.f;
+          }
+          psum += p0 + p1;
+          pk[i >> 1] = pack2<DT>(p0, p1);
+        }
+        tmem_st16(tmem_S + lane_addr + c * 16, pk);
+      }
+      l_sum += psum;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars.p_full);
+    }
+    // epilogue: O / l -> global
+    if (ok) ok = mbar_wait(&bars.o_full, 0, abort_flag);
+    if (ok) {
+      tc_fence_after();
+      const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+      const int hq = hk * rep + row % rep;
+      uint8_t* orow = rq.out + (((size_t)l * rq.sel_capacity + i_row) * m.Hq + hq) * (kD * 2);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld32(tmem_O + lane_addr + c * 32, r);
+        if (i_row < n_sel) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint4 w;
+            w.x = pack2<DT>(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
+            w.y = pack2<DT>(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+            w.z = pack2<DT>(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+            w.w = pack2<DT>(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + (c * 32 + i) * 2) = w;
+          }
+        }
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown (all roles)
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+  if (tid == 0 && s_abort) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
+}
+
+constexpr size_t kSmemBytes = 3 * kTileBytes + 1024;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+}  // namespace
+
+cudaError_t attention_tc_configure() {
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+    g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<KVB_DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attn_tc_kernel<KVB_DT_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+}
+
+// Host: the two tensor maps of one request (Q tile boxes, K/V block boxes), written to `out[0..1]`.
+int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity, const void* kv_buf, int T, void* out) {
+  if (!g_encode) return 1;
+  CUtensorMap* maps = static_cast<CUtensorMap*>(out);
+  const CUtensorMapDataType dt = m.dtype == KVB_DT_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16;
+  const int rep = m.Hq / m.Hkv;
+  const cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+  {  // Q: [L][cap][Hq][d] -> dims (d, Hq, cap, L); box = 64 x rep x TOK x 1 (128 rows of 128 bytes)
+    const cuuint64_t dims[4] = {(cuuint64_t)m.d, (cuuint64_t)m.Hq, (cuuint64_t)sel_capacity, (cuuint64_t)m.L};
+    const cuuint64_t strides[3] = {(cuuint64_t)m.d * 2, (cuuint64_t)m.Hq * m.d * 2, (cuuint64_t)sel_capacity * m.Hq * m.d * 2};
+    const cuuint32_t box[4] = {64, (cuuint32_t)rep, (cuuint32_t)(kRows / rep), 1};
+    if (g_encode(&maps[0], dt, 4, const_cast<void*>(q), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return 2;
+  }
+  {  // KV: [L][2][T][H][d] -> dims (d, H, T, 2, L); box = 64 x 1 x 128 x 1 x 1
+    const cuuint64_t dims[5] = {(cuuint64_t)m.d, (cuuint64_t)m.Hkv, (cuuint64_t)T, 2, (cuuint64_t)m.L};
+    const cuuint64_t strides[4] = {(cuuint64_t)m.d * 2, (cuuint64_t)m.Hkv * m.d * 2, (cuuint64_t)T * m.Hkv * m.d * 2,
+                                   (cuuint64_t)2 * T * m.Hkv * m.d * 2};
+    const cuuint32_t box[5] = {64, 1, (cuuint32_t)kBlockKeys, 1, 1};
+    if (g_encode(&maps[1], dt, 5, const_cast<void*>(kv_buf), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return 3;
+  }
+  return 0;
+}
+
+cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,
+                                float scale, uint32_t* status, cudaStream_t st) {
+  const unsigned grid = (unsigned)total_tiles * m.Hkv * m.L;
+  const float scale_log2 = scale * 1.4426950408889634f;
+  const CUtensorMap* mp = static_cast<const CUtensorMap*>(maps);
+  if (m.dtype == KVB_DT_BF16)
+    attn_tc_kernel<KVB_DT_BF16><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status);
+  else
+    attn_tc_kernel<KVB_DT_F16><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status);
+  return cudaGetLastError();
+}
+
+}  // namespace kvb

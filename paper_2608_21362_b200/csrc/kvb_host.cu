@@ -3,6 +3,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -34,6 +35,7 @@ struct kvb_ctx {
   int next_slot = 0;
   size_t arena_bytes = 0;
   bool acc_dirty = false;
+  bool attn_legacy = false;  // KVB_ATTN=mma selects the warp-level mma.sync kernel (debug aid)
   cudaStream_t last_stream = nullptr;
   int64_t launches = 0;
   char err[512] = {0};
@@ -206,6 +208,9 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, assemble_configure(smem_max));
   KVB_CUDA(c, topk_configure());
   KVB_CUDA(c, attention_mma_configure());
+  KVB_CUDA(c, attention_tc_configure());
+  const char* attn_env = getenv("KVB_ATTN");
+  c->attn_legacy = attn_env && strcmp(attn_env, "mma") == 0;
 
   const int half = m.d / 2;
   std::vector<double> inv(half);
@@ -215,7 +220,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, cudaMalloc(&c->cs_table, (size_t)limits->max_chunks_total * half * sizeof(float2)));
 
   const size_t a1 = sizeof(ChunkDesc) * (size_t)limits->max_chunks_total;
-  const size_t a2 = sizeof(ReqDesc) * (size_t)limits->max_requests + sizeof(SeamWindow) * (size_t)limits->max_chunks_total;
+  const size_t a2 = (sizeof(ReqDesc) + 256) * (size_t)limits->max_requests + 128 + sizeof(SeamWindow) * (size_t)limits->max_chunks_total;
   c->arena_bytes = ((a1 > a2 ? a1 : a2) + 255) & ~(size_t)255;
   KVB_CUDA(c, cudaMalloc(&c->arena_dev, c->arena_bytes));
   KVB_CUDA(c, cudaMallocHost(&c->staging, c->arena_bytes * kSlots));
@@ -395,6 +400,7 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
   if (slot_code >= 0) return slot_code;
   const int slot = -slot_code - 1;
   ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
+  const size_t maps_off = (sizeof(ReqDesc) * (size_t)n_req + 127) & ~(size_t)127;  // tensor maps: 2 x 128 bytes per request
   const int tok_per_tile = 128 / (c->model.Hq / c->model.Hkv);
   int tiles = 0;
   for (int r = 0; r < n_req; ++r) {
@@ -413,11 +419,19 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
     d.tile_offset = tiles;
     rd[r] = d;
     tiles += (s.sel_capacity + tok_per_tile - 1) / tok_per_tile;
+    if (!c->attn_legacy) {
+      const int e = attention_tc_encode_maps(c->dims, q[r], s.sel_capacity, reqs[r].kv_buf, reqs[r].T, host + maps_off + 256 * (size_t)r);
+      if (e != 0) return fail(c, KVB_ERR_CUDA, "request %d: tensor map encoding failed (%d)", r, e);
+    }
   }
-  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req, st);
+  const int up = upload(c, slot, host, maps_off + 256 * (size_t)n_req, st);
   if (up != KVB_OK) return up;
   c->last_stream = st;
-  KVB_CUDA(c, launch_attention_mma(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, tiles, c->dims, softmax_scale, st));
+  const ReqDesc* rd_dev = reinterpret_cast<const ReqDesc*>(c->arena_dev);
+  if (c->attn_legacy)
+    KVB_CUDA(c, launch_attention_mma(rd_dev, n_req, tiles, c->dims, softmax_scale, st));
+  else
+    KVB_CUDA(c, launch_attention_tc(rd_dev, c->arena_dev + maps_off, n_req, tiles, c->dims, softmax_scale, c->status_dev, st));
   c->launches += 1;
   return KVB_OK;
 }

@@ -79,6 +79,12 @@ cudaError_t launch_attention_mma(const ReqDesc* reqs, int n_req, int total_tiles
                                  cudaStream_t st);
 cudaError_t attention_mma_configure();
 
+cudaError_t attention_tc_configure();
+// Encodes the request's two TMA tensor maps (Q, KV) into out[0..255]; returns 0 on success.
+int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity, const void* kv_buf, int T, void* out);
+cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,
+                                float scale, uint32_t* status, cudaStream_t st);
+
 cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
                             cudaStream_t st);
 
