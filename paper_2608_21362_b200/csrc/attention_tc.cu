@@ -2,7 +2,7 @@
 //
 // One CTA per (layer, KV head, tile of selected tokens); a tile packs TOK = 128/rep selected
 // tokens times the rep = Hq/Hkv query heads sharing the KV head into the 128 rows of one
-// tcgen05.mma (M = 128).  Keys go by blocks of 128:
+// tcgen05.mma (M = 128).  Keys go by sub-blocks of 64, two streams alternating:
 //     S = Q K^T   tcgen05.mma, Q and K from shared memory (K-major, 128-byte swizzle), S in TMEM
 //     P = exp2(scale*S - m)  by 128 threads, one TMEM lane (row) each, written back over S as bf16
 //     O += P V    tcgen05.mma, P from TMEM, V from shared memory (MN-major), O in TMEM
@@ -27,10 +27,11 @@ namespace {
 
 constexpr int kThreads = 192;
 constexpr int kRows = 128;
-constexpr int kBlockKeys = 128;
+constexpr int kSubKeys = 64;                         // keys per sub-block (one stream's MMA N)
 constexpr int kD = 128;
 constexpr uint32_t kTileBytes = kRows * kD * 2;      // 32 KB: Q, K or V tile
-constexpr uint32_t kHalfBytes = kTileBytes / 2;      // one 64-element-wide TMA box
+constexpr uint32_t kHalfBytes = kTileBytes / 2;      // one 64-element-wide TMA box of Q (128 rows)
+constexpr uint32_t kSubBytes = kSubKeys * kD * 2;    // 16 KB: one stream's K or V sub-block
 constexpr uint32_t kTmemCols = 256;                  // S/P: columns 0..127, O: columns 128..255
 constexpr uint32_t kWaitLimit = 1u << 24;
 constexpr float kLazyThreshold = 8.0f;
@@ -148,16 +149,16 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return d;
 }
 
-// Instruction descriptor: float32 accumulate, A/B bf16 or fp16, M = 128, N = 128.
+// Instruction descriptor: float32 accumulate, A/B bf16 or fp16, M = 128, N = n.
 template <int DT>
-__device__ __forceinline__ uint32_t instr_desc(bool b_mn_major) {
+__device__ __forceinline__ uint32_t instr_desc(uint32_t n, bool b_mn_major) {
   const uint32_t fmt = DT == KVB_DT_BF16 ? 1u : 0u;
   uint32_t d = 0;
   d |= 1u << 4;                      // D format f32
   d |= fmt << 7;                     // A format
   d |= fmt << 10;                    // B format
   d |= (b_mn_major ? 1u : 0u) << 16; // B major: 0 = K, 1 = MN
-  d |= (128u >> 3) << 17;            // N
+  d |= (n >> 3) << 17;               // N
   d |= (128u >> 4) << 24;            // M
   return d;
 }
@@ -180,9 +181,13 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 struct __align__(8) Barriers {
-  uint64_t q_full, k_full, k_empty, v_full, v_empty, s_full, p_full, o_full;
+  uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], o_full;
 };
 
+// Keys are consumed in sub-blocks of 64, alternating between two streams x = sb & 1.  Each stream has
+// its own K and V buffers (16 KB each), its own S/P columns in TMEM and its own barriers, so while the
+// softmax threads work on one stream's scores the tensor core runs the other stream's P V and the
+// next Q K^T of the stream just consumed.  Both streams accumulate into the same O.
 template <int DT>
 __global__ void __launch_bounds__(kThreads, 2)
     attn_tc_kernel(const ReqDesc* __restrict__ reqs, const CUtensorMap* __restrict__ maps, int n_req, int total_tiles,
@@ -194,42 +199,48 @@ __global__ void __launch_bounds__(kThreads, 2)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int per_tile = m.Hkv * m.L;
+  const int rep = m.Hq / m.Hkv;
+  const int TOK = kRows / rep;
+  // CTA order: request, then (layer, KV head), then tiles from the longest down, so that CTAs resident
+  // together stream the same K/V planes (L2 reuse) and the long tiles start first.
   const int lin = blockIdx.x;
-  const int tile_flat = total_tiles - 1 - lin / per_tile;  // longest tiles first
-  const int hk = (lin % per_tile) % m.Hkv;
-  const int l = (lin % per_tile) / m.Hkv;
   int lo = 0, hi = n_req - 1;
   while (lo < hi) {
     const int mid = (lo + hi + 1) >> 1;
-    if (reqs[mid].tile_offset <= tile_flat) lo = mid; else hi = mid - 1;
+    if (reqs[mid].tile_offset * per_tile <= lin) lo = mid; else hi = mid - 1;
   }
   const ReqDesc rq = reqs[lo];
+  const int tiles_r = (rq.sel_capacity + TOK - 1) / TOK;
+  const int idx = lin - rq.tile_offset * per_tile;
+  const int lhk = idx / tiles_r;
+  const int tile = tiles_r - 1 - idx % tiles_r;
+  const int hk = lhk % m.Hkv;
+  const int l = lhk / m.Hkv;
   const CUtensorMap* map_q = maps + 2 * lo;
   const CUtensorMap* map_kv = maps + 2 * lo + 1;
-  const int rep = m.Hq / m.Hkv;
-  const int TOK = kRows / rep;
-  const int tile = tile_flat - rq.tile_offset;
   const int n_sel = min(*rq.n_sel, rq.sel_capacity);
   const int i_base = tile * TOK;
   if (i_base >= n_sel) return;  // uniform for the CTA, before anything is allocated
   const int T = rq.T;
   const int t_max = min(rq.sel[min(i_base + TOK, n_sel) - 1], T - 1);
-  const int nkb = t_max / kBlockKeys + 1;
+  const int nsb = t_max / kSubKeys + 1;  // 64-key sub-blocks to visit
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;
-  uint8_t* sK = smem + kTileBytes;
-  uint8_t* sV = smem + 2 * kTileBytes;
+  uint8_t* sQ = smem;                   // 128 rows: two 64-wide boxes of 16 KB
+  uint8_t* sK = smem + kTileBytes;      // stream x at + x * 16 KB: two 64-wide boxes of 8 KB (64 keys)
+  uint8_t* sV = smem + 2 * kTileBytes;  // same
   volatile uint32_t* abort_flag = &s_abort;
 
   if (tid == 0) {
     mbar_init(&bars.q_full, 1);
-    mbar_init(&bars.k_full, 1);
-    mbar_init(&bars.k_empty, 1);
-    mbar_init(&bars.v_full, 1);
-    mbar_init(&bars.v_empty, 1);
-    mbar_init(&bars.s_full, 1);
-    mbar_init(&bars.p_full, 128);
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(&bars.k_full[x], 1);
+      mbar_init(&bars.k_empty[x], 1);
+      mbar_init(&bars.v_full[x], 1);
+      mbar_init(&bars.v_empty[x], 1);
+      mbar_init(&bars.s_full[x], 1);
+      mbar_init(&bars.p_full[x], 128);
+    }
     mbar_init(&bars.o_full, 1);
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -242,7 +253,7 @@ __global__ void __launch_bounds__(kThreads, 2)
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = s_tmem_base;
-  const uint32_t tmem_S = tmem_base;        // also P (packed 16-bit pairs, columns 0..63)
+  const uint32_t tmem_S = tmem_base;        // stream x: columns 64x..64x+63 (P packed over the first 32 of them)
   const uint32_t tmem_O = tmem_base + 128;
 
   if (warp == 0) {
@@ -254,45 +265,60 @@ __global__ void __launch_bounds__(kThreads, 2)
       tma_load_4d(sQ, map_q, 0, hk * rep, i_base, l, &bars.q_full);
       tma_load_4d(sQ + kHalfBytes, map_q, 64, hk * rep, i_base, l, &bars.q_full);
       bool ok = true;
-      for (int j = 0; j < nkb && ok; ++j) {
-        if (j > 0) ok = mbar_wait(&bars.k_empty, (j - 1) & 1, abort_flag);
+      for (int sb = 0; sb < nsb && ok; ++sb) {
+        const int x = sb & 1;
+        const uint32_t prev = ((sb >> 1) & 1) ^ 1;  // parity of the use two sub-blocks ago
+        if (sb >= 2) ok = mbar_wait(&bars.k_empty[x], prev, abort_flag);
         if (!ok) break;
-        mbar_expect_tx(&bars.k_full, kTileBytes);
-        tma_load_5d(sK, map_kv, 0, hk, j * kBlockKeys, 0, l, &bars.k_full);
-        tma_load_5d(sK + kHalfBytes, map_kv, 64, hk, j * kBlockKeys, 0, l, &bars.k_full);
-        if (j > 0) ok = mbar_wait(&bars.v_empty, (j - 1) & 1, abort_flag);
+        mbar_expect_tx(&bars.k_full[x], kSubBytes);
+        tma_load_5d(sK + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
+        tma_load_5d(sK + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
+        if (sb >= 2) ok = mbar_wait(&bars.v_empty[x], prev, abort_flag);
         if (!ok) break;
-        mbar_expect_tx(&bars.v_full, kTileBytes);
-        tma_load_5d(sV, map_kv, 0, hk, j * kBlockKeys, 1, l, &bars.v_full);
-        tma_load_5d(sV + kHalfBytes, map_kv, 64, hk, j * kBlockKeys, 1, l, &bars.v_full);
+        mbar_expect_tx(&bars.v_full[x], kSubBytes);
+        tma_load_5d(sV + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
+        tma_load_5d(sV + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const uint32_t idesc_s = instr_desc<DT>(false);
-      const uint32_t idesc_pv = instr_desc<DT>(true);
+      const uint32_t idesc_s = instr_desc<DT>(kSubKeys, false);
+      const uint32_t idesc_pv = instr_desc<DT>(kD, true);
       const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
       bool ok = mbar_wait(&bars.q_full, 0, abort_flag);
-      for (int j = 0; j < nkb && ok; ++j) {
-        ok = mbar_wait(&bars.k_full, j & 1, abort_flag);
-        if (!ok) break;
+      auto issue_s = [&](int sb) {  // S_x = Q K_x^T, N = 64 keys
+        const int x = sb & 1;
+        if (!mbar_wait(&bars.k_full[x], (sb >> 1) & 1, abort_flag)) return false;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {  // 16 elements of d per step; 4 steps per 64-element box
-          const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-          mma_ss(tmem_S, smem_desc(q_addr + off, 16, 1024), smem_desc(k_addr + off, 16, 1024), idesc_s, ks > 0);
+          const uint32_t qo = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
+          const uint32_t ko = x * kSubBytes + (ks >> 2) * (kSubBytes / 2) + (ks & 3) * 32;
+          mma_ss(tmem_S + x * kSubKeys, smem_desc(q_addr + qo, 16, 1024), smem_desc(k_addr + ko, 16, 1024), idesc_s, ks > 0);
         }
-        tc_commit(&bars.s_full);
-        tc_commit(&bars.k_empty);
-        ok = mbar_wait(&bars.p_full, j & 1, abort_flag) && mbar_wait(&bars.v_full, j & 1, abort_flag);
-        if (!ok) break;
+        tc_commit(&bars.s_full[x]);
+        tc_commit(&bars.k_empty[x]);
+        return true;
+      };
+      auto issue_pv = [&](int sb) {  // O += P_x V_x, 64 keys = 4 steps of 16
+        const int x = sb & 1;
+        const uint32_t ph = (sb >> 1) & 1;
+        if (!mbar_wait(&bars.p_full[x], ph, abort_flag) || !mbar_wait(&bars.v_full[x], ph, abort_flag)) return false;
         tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {  // 16 keys per step = 2048 bytes of V; the two 64-wide halves of d are 16 KB apart
-          mma_ts(tmem_O, tmem_S + ks * 8, smem_desc(v_addr + ks * 2048, kHalfBytes, 1024), idesc_pv, (j > 0 || ks > 0));
+        for (int ks = 0; ks < 4; ++ks) {  // 16 keys = 2048 bytes of V; the two 64-wide halves of d are 8 KB apart
+          mma_ts(tmem_O, tmem_S + x * kSubKeys + ks * 8, smem_desc(v_addr + x * kSubBytes + ks * 2048, kSubBytes / 2, 1024), idesc_pv,
+                 (sb > 0 || ks > 0));
         }
-        tc_commit(&bars.v_empty);
+        tc_commit(&bars.v_empty[x]);
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      if (ok && nsb > 1) ok = issue_s(1);
+      for (int sb = 0; sb < nsb && ok; ++sb) {
+        ok = issue_pv(sb);
+        if (ok && sb + 2 < nsb) ok = issue_s(sb + 2);
       }
       if (ok) tc_commit(&bars.o_full);
     }
@@ -308,38 +334,41 @@ __global__ void __launch_bounds__(kThreads, 2)
     for (int o = 16; o >= 1; o >>= 1) warp_tmin = min(warp_tmin, __shfl_xor_sync(0xffffffffu, warp_tmin, o));
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = true;
-    for (int j = 0; j < nkb; ++j) {
-      ok = mbar_wait(&bars.s_full, j & 1, abort_flag);
+    for (int sb = 0; sb < nsb; ++sb) {
+      const int x = sb & 1;
+      ok = mbar_wait(&bars.s_full[x], (sb >> 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after();
-      const int key0 = j * kBlockKeys;
-      const bool need_mask = key0 + kBlockKeys - 1 > warp_tmin;
-      // pass 1: block maximum of this row
-      float bm = -INFINITY;
+      const int key0 = sb * kSubKeys;
+      const bool need_mask = key0 + kSubKeys - 1 > warp_tmin;
+      const uint32_t s_addr = tmem_S + lane_addr + x * kSubKeys;
+      uint32_t r0[32], r1[32];
+      tmem_ld32(s_addr, r0);
+      tmem_ld32(s_addr + 32, r1);
+      if (need_mask) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem_S + lane_addr + c * 32, r);
-        if (need_mask) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (key0 + c * 32 + i <= t_row) bm = fmaxf(bm, __uint_as_float(r[i]));
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) bm = fmaxf(bm, __uint_as_float(r[i]));
+        for (int i = 0; i < 32; ++i) {
+          if (key0 + i > t_row) r0[i] = 0xFF800000u;  // -inf
+          if (key0 + 32 + i > t_row) r1[i] = 0xFF800000u;
         }
       }
+      float bm = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 32; ++i) bm = fmaxf(bm, fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])));
       bm *= scale_log2;  // scale_log2 > 0, so the maximum commutes with the scaling
       // lazy reference maximum; O rows are rescaled only when the reference moves
       float factor = 1.f;
-      if (bm > m_ref + kLazyThreshold || m_ref == -INFINITY) {
-        if (bm > -INFINITY) {
-          factor = m_ref == -INFINITY ? 0.f : exp2f(m_ref - bm);
-          m_ref = bm;
-        }
+      if ((bm > m_ref + kLazyThreshold || m_ref == -INFINITY) && bm > -INFINITY) {
+        factor = m_ref == -INFINITY ? 0.f : fast_exp2(m_ref - bm);
+        m_ref = bm;
       }
-      const bool rescale = j > 0 && __any_sync(0xffffffffu, factor != 1.f);
-      if (rescale) {  // PV of the previous block is complete: S of this block was issued after it
+      const bool rescale = sb > 0 && __any_sync(0xffffffffu, factor != 1.f);
+      if (rescale) {
+        // no P V may be accumulating into O: the previous sub-block's must have completed, and the
+        // next one cannot start before this thread has arrived on p_full
+        ok = mbar_wait(&bars.v_empty[(sb - 1) & 1], ((sb - 1) >> 1) & 1, abort_flag);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        tc_fence_after();
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           uint32_t r[32];
@@ -351,30 +380,24 @@ __global__ void __launch_bounds__(kThreads, 2)
       }
       l_sum *= factor;
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
-      // pass 2: P = exp2(scale*S - m), packed to 16 bits over the S columns already consumed
+      // P = exp2(scale*S - m), packed to 16 bits over the first half of this stream's S columns
+      uint32_t pk[32];
       float psum = 0.f;
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem_S + lane_addr + c * 32, r);
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_use));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_use));
-          if (need_mask) {
-            if (key0 + c * 32 + i > t_row) p0 = 0.f;
-            if (key0 + c * 32 + i + 1 > t_row) p1 = 0.f;
-          }
-          psum += p0 + p1;
-          pk[i >> 1] = pack2<DT>(p0, p1);
-        }
-        tmem_st16(tmem_S + lane_addr + c * 16, pk);
+      for (int i = 0; i < 32; i += 2) {
+        const float p0 = fast_exp2(fmaf(__uint_as_float(r0[i]), scale_log2, -m_use));
+        const float p1 = fast_exp2(fmaf(__uint_as_float(r0[i + 1]), scale_log2, -m_use));
+        const float p2 = fast_exp2(fmaf(__uint_as_float(r1[i]), scale_log2, -m_use));
+        const float p3 = fast_exp2(fmaf(__uint_as_float(r1[i + 1]), scale_log2, -m_use));
+        psum += (p0 + p1) + (p2 + p3);
+        pk[i >> 1] = pack2<DT>(p0, p1);
+        pk[16 + (i >> 1)] = pack2<DT>(p2, p3);
       }
       l_sum += psum;
+      tmem_st32(s_addr, pk);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bars.p_full);
+      mbar_arrive(&bars.p_full[x]);
     }
     // epilogue: O / l -> global
     if (ok) ok = mbar_wait(&bars.o_full, 0, abort_flag);
@@ -450,11 +473,11 @@ int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity
                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return 2;
   }
-  {  // KV: [L][2][T][H][d] -> dims (d, H, T, 2, L); box = 64 x 1 x 128 x 1 x 1
+  {  // KV: [L][2][T][H][d] -> dims (d, H, T, 2, L); box = 64 x 1 x 64 keys x 1 x 1
     const cuuint64_t dims[5] = {(cuuint64_t)m.d, (cuuint64_t)m.Hkv, (cuuint64_t)T, 2, (cuuint64_t)m.L};
     const cuuint64_t strides[4] = {(cuuint64_t)m.d * 2, (cuuint64_t)m.Hkv * m.d * 2, (cuuint64_t)T * m.Hkv * m.d * 2,
                                    (cuuint64_t)2 * T * m.Hkv * m.d * 2};
-    const cuuint32_t box[5] = {64, 1, (cuuint32_t)kBlockKeys, 1, 1};
+    const cuuint32_t box[5] = {64, 1, (cuuint32_t)kSubKeys, 1, 1};
     if (g_encode(&maps[1], dt, 5, const_cast<void*>(kv_buf), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
       return 3;
