@@ -35,6 +35,7 @@ constexpr uint32_t kSubBytes = kSubKeys * kD * 2;    // 16 KB: one stream's K or
 constexpr uint32_t kTmemCols = 256;                  // S/P: columns 0..127, O: columns 128..255
 constexpr uint32_t kWaitLimit = 1u << 24;
 constexpr float kLazyThreshold = 8.0f;
+constexpr bool kPolyExp = false;  // one exp2 in four goes to the FMA pipe
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -169,6 +170,43 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// 2^x on the FMA and integer pipes (no MUFU): round to the nearest integer with the 1.5*2^23 trick,
+// a cubic for 2^f on [-0.5, 0.5] (relative error 7.5e-5, far below the 16-bit rounding of P), and
+// the integer part added into the exponent field.  Used for a fraction of the scores so that the
+// 16-per-clock special-function unit is not the limiter.
+__device__ __forceinline__ float poly_exp2(float x) {
+  x = fmaxf(x, -125.f);
+  const float t = x + 12582912.f;
+  const float f = x - (t - 12582912.f);
+  float p = fmaf(0.05517165f, f, 0.24261113f);
+  p = fmaf(p, f, 0.69326097f);
+  p = fmaf(p, f, 0.99992806f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+// Packed float32 pairs (one instruction for two lanes of work) and the three-input maximum.
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t d, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(d)); }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 template <int DT>
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
   if (DT == KVB_DT_BF16) {
@@ -264,20 +302,33 @@ __global__ void __launch_bounds__(kThreads, 2)
       mbar_expect_tx(&bars.q_full, kTileBytes);
       tma_load_4d(sQ, map_q, 0, hk * rep, i_base, l, &bars.q_full);
       tma_load_4d(sQ + kHalfBytes, map_q, 64, hk * rep, i_base, l, &bars.q_full);
-      bool ok = true;
-      for (int sb = 0; sb < nsb && ok; ++sb) {
+      // Loads are issued in the order their buffers come free: K(sb+2) as soon as S(sb) has read
+      // K(sb), V(sb) as soon as P V(sb-2) has read V(sb-2):  K0 K1 | V0 K2 | V1 K3 | ...
+      auto load_k = [&](int sb) {
         const int x = sb & 1;
-        const uint32_t prev = ((sb >> 1) & 1) ^ 1;  // parity of the use two sub-blocks ago
-        if (sb >= 2) ok = mbar_wait(&bars.k_empty[x], prev, abort_flag);
-        if (!ok) break;
         mbar_expect_tx(&bars.k_full[x], kSubBytes);
         tma_load_5d(sK + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
         tma_load_5d(sK + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
-        if (sb >= 2) ok = mbar_wait(&bars.v_empty[x], prev, abort_flag);
-        if (!ok) break;
+      };
+      auto load_v = [&](int sb) {
+        const int x = sb & 1;
         mbar_expect_tx(&bars.v_full[x], kSubBytes);
         tma_load_5d(sV + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
         tma_load_5d(sV + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
+      };
+      load_k(0);
+      if (nsb > 1) load_k(1);
+      bool ok = true;
+      for (int sb = 0; sb < nsb && ok; ++sb) {
+        const int x = sb & 1;
+        if (sb >= 2) ok = mbar_wait(&bars.v_empty[x], ((sb >> 1) & 1) ^ 1, abort_flag);  // P V(sb-2) done
+        if (!ok) break;
+        load_v(sb);
+        if (sb + 2 < nsb) {
+          ok = mbar_wait(&bars.k_empty[x], (sb >> 1) & 1, abort_flag);  // S(sb) done
+          if (!ok) break;
+          load_k(sb + 2);
+        }
       }
     }
   } else if (warp == 1) {
@@ -287,15 +338,20 @@ __global__ void __launch_bounds__(kThreads, 2)
       const uint32_t idesc_pv = instr_desc<DT>(kD, true);
       const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
       bool ok = mbar_wait(&bars.q_full, 0, abort_flag);
+      // descriptors differ only in their start-address field (units of 16 bytes, low word)
+      const uint64_t q_desc = smem_desc(q_addr, 16, 1024);
+      const uint64_t k_desc = smem_desc(k_addr, 16, 1024);
+      const uint64_t v_desc = smem_desc(v_addr, kSubBytes / 2, 1024);
       auto issue_s = [&](int sb) {  // S_x = Q K_x^T, N = 64 keys
         const int x = sb & 1;
         if (!mbar_wait(&bars.k_full[x], (sb >> 1) & 1, abort_flag)) return false;
         tc_fence_after();
+        const uint64_t kd = k_desc + (uint64_t)(x * (kSubBytes >> 4));
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {  // 16 elements of d per step; 4 steps per 64-element box
           const uint32_t qo = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-          const uint32_t ko = x * kSubBytes + (ks >> 2) * (kSubBytes / 2) + (ks & 3) * 32;
-          mma_ss(tmem_S + x * kSubKeys, smem_desc(q_addr + qo, 16, 1024), smem_desc(k_addr + ko, 16, 1024), idesc_s, ks > 0);
+          const uint32_t ko = (ks >> 2) * (kSubBytes / 2) + (ks & 3) * 32;
+          mma_ss(tmem_S + x * kSubKeys, q_desc + (qo >> 4), kd + (ko >> 4), idesc_s, ks > 0);
         }
         tc_commit(&bars.s_full[x]);
         tc_commit(&bars.k_empty[x]);
@@ -307,9 +363,10 @@ __global__ void __launch_bounds__(kThreads, 2)
         if (!mbar_wait(&bars.p_full[x], ph, abort_flag) || !mbar_wait(&bars.v_full[x], ph, abort_flag)) return false;
         tc_fence_after();
 #pragma unroll
+        const uint64_t vd = v_desc + (uint64_t)(x * (kSubBytes >> 4));
+#pragma unroll
         for (int ks = 0; ks < 4; ++ks) {  // 16 keys = 2048 bytes of V; the two 64-wide halves of d are 8 KB apart
-          mma_ts(tmem_O, tmem_S + x * kSubKeys + ks * 8, smem_desc(v_addr + x * kSubBytes + ks * 2048, kSubBytes / 2, 1024), idesc_pv,
-                 (sb > 0 || ks > 0));
+          mma_ts(tmem_O, tmem_S + x * kSubKeys + ks * 8, vd + (ks * 2048 >> 4), idesc_pv, (sb > 0 || ks > 0));
         }
         tc_commit(&bars.v_empty[x]);
         return true;
@@ -352,10 +409,17 @@ __global__ void __launch_bounds__(kThreads, 2)
           if (key0 + 32 + i > t_row) r1[i] = 0xFF800000u;
         }
       }
-      float bm = -INFINITY;
+      float mx[4] = {__uint_as_float(r0[0]), __uint_as_float(r0[1]), __uint_as_float(r1[0]), __uint_as_float(r1[1])};
 #pragma unroll
-      for (int i = 0; i < 32; ++i) bm = fmaxf(bm, fmaxf(__uint_as_float(r0[i]), __uint_as_float(r1[i])));
-      bm *= scale_log2;  // scale_log2 > 0, so the maximum commutes with the scaling
+      for (int i = 2; i < 32; i += 4) {
+        mx[0] = fmax3(mx[0], __uint_as_float(r0[i]), __uint_as_float(r0[i + 1]));
+        mx[2] = fmax3(mx[2], __uint_as_float(r1[i]), __uint_as_float(r1[i + 1]));
+        if (i + 2 < 32) {
+          mx[1] = fmax3(mx[1], __uint_as_float(r0[i + 2]), __uint_as_float(r0[i + 3]));
+          mx[3] = fmax3(mx[3], __uint_as_float(r1[i + 2]), __uint_as_float(r1[i + 3]));
+        }
+      }
+      const float bm = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0 commutes with max
       // lazy reference maximum; O rows are rescaled only when the reference moves
       float factor = 1.f;
       if ((bm > m_ref + kLazyThreshold || m_ref == -INFINITY) && bm > -INFINITY) {
@@ -382,18 +446,25 @@ __global__ void __launch_bounds__(kThreads, 2)
       const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
       // P = exp2(scale*S - m), packed to 16 bits over the first half of this stream's S columns
       uint32_t pk[32];
-      float psum = 0.f;
+      const uint64_t scale2 = f2_pack(scale_log2, scale_log2), negm2 = f2_pack(-m_use, -m_use);
+      uint64_t ps2[4] = {0ull, 0ull, 0ull, 0ull};  // packed partial sums (bit pattern of +0, +0)
 #pragma unroll
       for (int i = 0; i < 32; i += 2) {
-        const float p0 = fast_exp2(fmaf(__uint_as_float(r0[i]), scale_log2, -m_use));
-        const float p1 = fast_exp2(fmaf(__uint_as_float(r0[i + 1]), scale_log2, -m_use));
-        const float p2 = fast_exp2(fmaf(__uint_as_float(r1[i]), scale_log2, -m_use));
-        const float p3 = fast_exp2(fmaf(__uint_as_float(r1[i + 1]), scale_log2, -m_use));
-        psum += (p0 + p1) + (p2 + p3);
+        float a0, a1, a2, a3;
+        f2_unpack(f2_fma(f2_pack(__uint_as_float(r0[i]), __uint_as_float(r0[i + 1])), scale2, negm2), a0, a1);
+        f2_unpack(f2_fma(f2_pack(__uint_as_float(r1[i]), __uint_as_float(r1[i + 1])), scale2, negm2), a2, a3);
+        const float p0 = fast_exp2(a0), p1 = fast_exp2(a1), p2 = fast_exp2(a2);
+        const float p3 = kPolyExp ? poly_exp2(a3) : fast_exp2(a3);
+        ps2[(i >> 1) & 1] = f2_add(ps2[(i >> 1) & 1], f2_pack(p0, p1));
+        ps2[2 + ((i >> 1) & 1)] = f2_add(ps2[2 + ((i >> 1) & 1)], f2_pack(p2, p3));
         pk[i >> 1] = pack2<DT>(p0, p1);
         pk[16 + (i >> 1)] = pack2<DT>(p2, p3);
       }
-      l_sum += psum;
+      {
+        float lo, hi;
+        f2_unpack(f2_add(f2_add(ps2[0], ps2[1]), f2_add(ps2[2], ps2[3])), lo, hi);
+        l_sum += lo + hi;
+      }
       tmem_st32(s_addr, pk);
       tmem_wait_st();
       tc_fence_before();
