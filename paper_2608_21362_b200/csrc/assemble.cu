@@ -14,6 +14,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "f32x2.cuh"
 #include "kvb_internal.h"
 
 namespace kvb {
@@ -60,14 +61,15 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                : "memory");
 }
 
-// byte k of x -> float, exactly: place it in the mantissa of 2^23 and subtract 2^23
+// byte k of x in the low mantissa bits of 2^23: the float 2^23 + q
 template <int K>
-__device__ __forceinline__ float byte_to_float(uint32_t x) {
-  return __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650u + K)) - 8388608.0f;
+__device__ __forceinline__ float byte_magic(uint32_t x) {
+  return __uint_as_float(__byte_perm(x, 0x4B000000u, 0x7650u + K));
 }
+// nibble k of a 16-bit word in the top mantissa bits of 16.0: the float 16 + q
 template <int K>
-__device__ __forceinline__ float nibble_to_float(uint32_t x) {
-  return __uint_as_float(((x >> (4 * K)) & 0xFu) | 0x4B000000u) - 8388608.0f;
+__device__ __forceinline__ float nibble_magic(uint32_t x) {
+  return __uint_as_float(((x << (19 - 4 * K)) & 0x00780000u) | 0x41800000u);
 }
 
 template <typename T>
@@ -78,8 +80,8 @@ struct Pack<__nv_bfloat16> {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
   }
-  static __device__ __forceinline__ float2 unpack(uint32_t x) {
-    return make_float2(__uint_as_float(x << 16), __uint_as_float(x & 0xFFFF0000u));
+  static __device__ __forceinline__ uint64_t unpack2(uint32_t x) {
+    return f2_pack(__uint_as_float(x << 16), __uint_as_float(x & 0xFFFF0000u));
   }
 };
 template <>
@@ -88,15 +90,18 @@ struct Pack<__half> {
     __half2 v = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
   }
-  static __device__ __forceinline__ float2 unpack(uint32_t x) {
-    return __half22float2(*reinterpret_cast<__half2*>(&x));
+  static __device__ __forceinline__ uint64_t unpack2(uint32_t x) {
+    const float2 t = __half22float2(*reinterpret_cast<__half2*>(&x));
+    return f2_pack(t.x, t.y);
   }
 };
 
 template <typename OutT>
-__device__ __forceinline__ void store4(OutT* p, const float (&v)[4]) {
-  uint2 w = make_uint2(Pack<OutT>::two(v[0], v[1]), Pack<OutT>::two(v[2], v[3]));
-  *reinterpret_cast<uint2*>(p) = w;
+__device__ __forceinline__ void store4(OutT* p, const uint64_t (&v)[2]) {
+  float a, b, c, e;
+  f2_unpack(v[0], a, b);
+  f2_unpack(v[1], c, e);
+  *reinterpret_cast<uint2*>(p) = make_uint2(Pack<OutT>::two(a, b), Pack<OutT>::two(c, e));
 }
 
 __device__ __forceinline__ void copy_rows(uint8_t* dst, const uint8_t* src, size_t bytes, int tid) {
@@ -207,9 +212,36 @@ __global__ void __launch_bounds__(kThreads, 3)
   if (meta_bytes) ok = mbar_wait(&bars[0], 0);
   int ready_part = -1;
 
+  // Codes become floats without a conversion instruction: an 8-bit code goes into the low mantissa
+  // bits of 2^23 (value 2^23 + q, then one exact subtraction, done on packed pairs); a 4-bit code
+  // goes into the top mantissa bits of 16.0 (value 16 + q) and the 16 is folded into the constant
+  // term.  All affine arithmetic runs on packed float32 pairs.
+  const uint64_t neg_magic2 = f2_pack(-8388608.0f, -8388608.0f);
+  auto load_codes = [&](int u, uint64_t (&ql)[2], uint64_t (&qh)[2]) {
+    if (bits == 8) {
+      const uint8_t* row = s_codes + (size_t)u * d;
+      const uint32_t xa = *reinterpret_cast<const uint32_t*>(row + off_a + 4 * ln);
+      const uint32_t xb = *reinterpret_cast<const uint32_t*>(row + off_b + 4 * ln);
+      const uint32_t xl = s ? xb : xa, xh = s ? xa : xb;
+      ql[0] = f2_add(f2_pack(byte_magic<0>(xl), byte_magic<1>(xl)), neg_magic2);
+      ql[1] = f2_add(f2_pack(byte_magic<2>(xl), byte_magic<3>(xl)), neg_magic2);
+      qh[0] = f2_add(f2_pack(byte_magic<0>(xh), byte_magic<1>(xh)), neg_magic2);
+      qh[1] = f2_add(f2_pack(byte_magic<2>(xh), byte_magic<3>(xh)), neg_magic2);
+    } else {
+      const uint8_t* row = s_codes + (size_t)u * (d / 2);
+      const uint32_t xl = *reinterpret_cast<const uint16_t*>(row + 2 * ln);
+      const uint32_t xh = *reinterpret_cast<const uint16_t*>(row + 32 + 2 * ln);
+      ql[0] = f2_pack(nibble_magic<0>(xl), nibble_magic<1>(xl));
+      ql[1] = f2_pack(nibble_magic<2>(xl), nibble_magic<3>(xl));
+      qh[0] = f2_pack(nibble_magic<0>(xh), nibble_magic<1>(xh));
+      qh[1] = f2_pack(nibble_magic<2>(xh), nibble_magic<3>(xh));
+    }
+  };
+  const float bias = bits == 4 ? 16.f : 0.f;  // what the 4-bit unpacking adds to every code
+
   if (!kv) {
     // ------------------------------ keys
-    float A_lo[4], B_lo[4], C_lo[4], A_hi[4], B_hi[4], C_hi[4];
+    uint64_t A_lo[2], B_lo[2], C_lo[2], A_hi[2], B_hi[2], C_hi[2];
     float cs_c[4], cs_s[4];
     {
       const float4* p = reinterpret_cast<const float4*>(cs_table + (size_t)ci * (d / 2) + 4 * ln);
@@ -217,6 +249,9 @@ __global__ void __launch_bounds__(kThreads, 3)
       cs_c[0] = a.x, cs_s[0] = a.y, cs_c[1] = a.z, cs_s[1] = a.w;
       cs_c[2] = b.x, cs_s[2] = b.y, cs_c[3] = b.z, cs_s[3] = b.w;
     }
+    const uint64_t c2[2] = {f2_pack(cs_c[0], cs_c[1]), f2_pack(cs_c[2], cs_c[3])};
+    const uint64_t s2[2] = {f2_pack(cs_s[0], cs_s[1]), f2_pack(cs_s[2], cs_s[3])};
+    const uint64_t ns2[2] = {f2_pack(-cs_s[0], -cs_s[1]), f2_pack(-cs_s[2], -cs_s[3])};
     int cur_group = -1;
 #pragma unroll 2
     for (int tt = 0; tt < tok_per; ++tt) {
@@ -229,63 +264,52 @@ __global__ void __launch_bounds__(kThreads, 3)
       if (!ok) break;
       const int u = t * H + h;
       OutT* orow = dst + (size_t)u * d;
-      float ql[4], qh[4];
+      uint64_t ol[2], oh[2];
       if (bits == 16) {
         const uint8_t* row = s_codes + (size_t)u * (d * 2);
-        uint2 a = *reinterpret_cast<const uint2*>(row + 8 * ln);
-        uint2 b = *reinterpret_cast<const uint2*>(row + 128 + 8 * ln);
-        float2 f;
-        f = Pack<OutT>::unpack(a.x), ql[0] = f.x, ql[1] = f.y;
-        f = Pack<OutT>::unpack(a.y), ql[2] = f.x, ql[3] = f.y;
-        f = Pack<OutT>::unpack(b.x), qh[0] = f.x, qh[1] = f.y;
-        f = Pack<OutT>::unpack(b.y), qh[2] = f.x, qh[3] = f.y;
-        float ol[4], oh[4];
+        const uint2 a = *reinterpret_cast<const uint2*>(row + 8 * ln);
+        const uint2 b = *reinterpret_cast<const uint2*>(row + 128 + 8 * ln);
+        const uint64_t xl[2] = {Pack<OutT>::unpack2(a.x), Pack<OutT>::unpack2(a.y)};
+        const uint64_t xh[2] = {Pack<OutT>::unpack2(b.x), Pack<OutT>::unpack2(b.y)};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          ol[i] = fmaf(ql[i], cs_c[i], -(qh[i] * cs_s[i]));
-          oh[i] = fmaf(qh[i], cs_c[i], ql[i] * cs_s[i]);
+        for (int i = 0; i < 2; ++i) {
+          ol[i] = f2_fma(xl[i], c2[i], f2_mul(xh[i], ns2[i]));
+          oh[i] = f2_fma(xh[i], c2[i], f2_mul(xl[i], s2[i]));
         }
-        store4(orow + 4 * ln, ol);
-        store4(orow + 64 + 4 * ln, oh);
-        continue;
-      }
-      const int g = (tb + t) / group_tokens - g_first;
-      if (g != cur_group) {
-        cur_group = g;
-        const float* mlo = s_meta + ((size_t)(g * H + h) * d + 4 * ln) * 2;
-        const float4 a0 = *reinterpret_cast<const float4*>(mlo), a1 = *reinterpret_cast<const float4*>(mlo + 4);
-        const float4 b0 = *reinterpret_cast<const float4*>(mlo + 128), b1 = *reinterpret_cast<const float4*>(mlo + 132);
-        const float sl[4] = {a0.x, a0.z, a1.x, a1.z}, ml[4] = {a0.y, a0.w, a1.y, a1.w};
-        const float sh[4] = {b0.x, b0.z, b1.x, b1.z}, mh[4] = {b0.y, b0.w, b1.y, b1.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          A_lo[i] = sl[i] * cs_c[i];
-          B_lo[i] = -(sh[i] * cs_s[i]);
-          C_lo[i] = fmaf(ml[i], cs_c[i], -(mh[i] * cs_s[i]));
-          A_hi[i] = sh[i] * cs_c[i];
-          B_hi[i] = sl[i] * cs_s[i];
-          C_hi[i] = fmaf(mh[i], cs_c[i], ml[i] * cs_s[i]);
-        }
-      }
-      if (bits == 8) {
-        const uint8_t* row = s_codes + (size_t)u * d;
-        const uint32_t xa = *reinterpret_cast<const uint32_t*>(row + off_a + 4 * ln);
-        const uint32_t xb = *reinterpret_cast<const uint32_t*>(row + off_b + 4 * ln);
-        const uint32_t xl = s ? xb : xa, xh = s ? xa : xb;
-        ql[0] = byte_to_float<0>(xl), ql[1] = byte_to_float<1>(xl), ql[2] = byte_to_float<2>(xl), ql[3] = byte_to_float<3>(xl);
-        qh[0] = byte_to_float<0>(xh), qh[1] = byte_to_float<1>(xh), qh[2] = byte_to_float<2>(xh), qh[3] = byte_to_float<3>(xh);
       } else {
-        const uint8_t* row = s_codes + (size_t)u * (d / 2);
-        const uint32_t xl = *reinterpret_cast<const uint16_t*>(row + 2 * ln);
-        const uint32_t xh = *reinterpret_cast<const uint16_t*>(row + 32 + 2 * ln);
-        ql[0] = nibble_to_float<0>(xl), ql[1] = nibble_to_float<1>(xl), ql[2] = nibble_to_float<2>(xl), ql[3] = nibble_to_float<3>(xl);
-        qh[0] = nibble_to_float<0>(xh), qh[1] = nibble_to_float<1>(xh), qh[2] = nibble_to_float<2>(xh), qh[3] = nibble_to_float<3>(xh);
-      }
-      float ol[4], oh[4];
+        const int g = (tb + t) / group_tokens - g_first;
+        if (g != cur_group) {
+          cur_group = g;
+          const float* mlo = s_meta + ((size_t)(g * H + h) * d + 4 * ln) * 2;
+          const float4 a0 = *reinterpret_cast<const float4*>(mlo), a1 = *reinterpret_cast<const float4*>(mlo + 4);
+          const float4 b0 = *reinterpret_cast<const float4*>(mlo + 128), b1 = *reinterpret_cast<const float4*>(mlo + 132);
+          const float sl[4] = {a0.x, a0.z, a1.x, a1.z}, ml[4] = {a0.y, a0.w, a1.y, a1.w};
+          const float sh[4] = {b0.x, b0.z, b1.x, b1.z}, mh[4] = {b0.y, b0.w, b1.y, b1.w};
+          float al[4], bl[4], cl[4], ah[4], bh[4], ch[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        ol[i] = fmaf(A_lo[i], ql[i], fmaf(B_lo[i], qh[i], C_lo[i]));
-        oh[i] = fmaf(A_hi[i], qh[i], fmaf(B_hi[i], ql[i], C_hi[i]));
+          for (int i = 0; i < 4; ++i) {
+            al[i] = sl[i] * cs_c[i];
+            bl[i] = -(sh[i] * cs_s[i]);
+            cl[i] = fmaf(ml[i], cs_c[i], -(mh[i] * cs_s[i]));
+            ah[i] = sh[i] * cs_c[i];
+            bh[i] = sl[i] * cs_s[i];
+            ch[i] = fmaf(mh[i], cs_c[i], ml[i] * cs_s[i]);
+            cl[i] = fmaf(-bias, al[i] + bl[i], cl[i]);
+            ch[i] = fmaf(-bias, ah[i] + bh[i], ch[i]);
+          }
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            A_lo[i] = f2_pack(al[2 * i], al[2 * i + 1]), B_lo[i] = f2_pack(bl[2 * i], bl[2 * i + 1]), C_lo[i] = f2_pack(cl[2 * i], cl[2 * i + 1]);
+            A_hi[i] = f2_pack(ah[2 * i], ah[2 * i + 1]), B_hi[i] = f2_pack(bh[2 * i], bh[2 * i + 1]), C_hi[i] = f2_pack(ch[2 * i], ch[2 * i + 1]);
+          }
+        }
+        uint64_t ql[2], qh[2];
+        load_codes(u, ql, qh);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          ol[i] = f2_fma(A_lo[i], ql[i], f2_fma(B_lo[i], qh[i], C_lo[i]));
+          oh[i] = f2_fma(A_hi[i], qh[i], f2_fma(B_hi[i], ql[i], C_hi[i]));
+        }
       }
       store4(orow + 4 * ln, ol);
       store4(orow + 64 + 4 * ln, oh);
@@ -303,33 +327,23 @@ __global__ void __launch_bounds__(kThreads, 3)
       if (!ok) break;
       const int u = t * H + h;
       OutT* orow = dst + (size_t)u * d;
-      float ql[4], qh[4];
       float s_lo, m_lo, s_hi, m_hi;
       if (bits == 8) {
         const float2 sm = *reinterpret_cast<const float2*>(s_meta + (size_t)u * 2);
         s_lo = s_hi = sm.x, m_lo = m_hi = sm.y;
-        const uint8_t* row = s_codes + (size_t)u * d;
-        const uint32_t xa = *reinterpret_cast<const uint32_t*>(row + off_a + 4 * ln);
-        const uint32_t xb = *reinterpret_cast<const uint32_t*>(row + off_b + 4 * ln);
-        const uint32_t xl = s ? xb : xa, xh = s ? xa : xb;
-        ql[0] = byte_to_float<0>(xl), ql[1] = byte_to_float<1>(xl), ql[2] = byte_to_float<2>(xl), ql[3] = byte_to_float<3>(xl);
-        qh[0] = byte_to_float<0>(xh), qh[1] = byte_to_float<1>(xh), qh[2] = byte_to_float<2>(xh), qh[3] = byte_to_float<3>(xh);
       } else {
         const int g_lo = (4 * ln) / m.int4_group, g_hi = (64 + 4 * ln) / m.int4_group;
         const float2 a = *reinterpret_cast<const float2*>(s_meta + ((size_t)u * G + g_lo) * 2);
         const float2 b = *reinterpret_cast<const float2*>(s_meta + ((size_t)u * G + g_hi) * 2);
-        s_lo = a.x, m_lo = a.y, s_hi = b.x, m_hi = b.y;
-        const uint8_t* row = s_codes + (size_t)u * (d / 2);
-        const uint32_t xl = *reinterpret_cast<const uint16_t*>(row + 2 * ln);
-        const uint32_t xh = *reinterpret_cast<const uint16_t*>(row + 32 + 2 * ln);
-        ql[0] = nibble_to_float<0>(xl), ql[1] = nibble_to_float<1>(xl), ql[2] = nibble_to_float<2>(xl), ql[3] = nibble_to_float<3>(xl);
-        qh[0] = nibble_to_float<0>(xh), qh[1] = nibble_to_float<1>(xh), qh[2] = nibble_to_float<2>(xh), qh[3] = nibble_to_float<3>(xh);
+        s_lo = a.x, m_lo = fmaf(-bias, a.x, a.y), s_hi = b.x, m_hi = fmaf(-bias, b.x, b.y);
       }
-      float ol[4], oh[4];
+      uint64_t ql[2], qh[2], ol[2], oh[2];
+      load_codes(u, ql, qh);
+      const uint64_t sl2 = f2_pack(s_lo, s_lo), ml2 = f2_pack(m_lo, m_lo), sh2 = f2_pack(s_hi, s_hi), mh2 = f2_pack(m_hi, m_hi);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        ol[i] = fmaf(ql[i], s_lo, m_lo);
-        oh[i] = fmaf(qh[i], s_hi, m_hi);
+      for (int i = 0; i < 2; ++i) {
+        ol[i] = f2_fma(ql[i], sl2, ml2);
+        oh[i] = f2_fma(qh[i], sh2, mh2);
       }
       store4(orow + 4 * ln, ol);
       store4(orow + 64 + 4 * ln, oh);

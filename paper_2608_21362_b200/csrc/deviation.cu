@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "f32x2.cuh"
 #include "kvb_internal.h"
 
 namespace kvb {
@@ -21,35 +22,30 @@ constexpr int kThreads = 256;
 constexpr int kTileTokens = 64;
 constexpr float kFixScale = 1099511627776.0f;  // 2^40
 
+// One 32-bit word holds two 16-bit values: unpack them into a packed float32 pair.
 template <int DT>
-__device__ __forceinline__ void unpack8(const uint4& v, float (&f)[8]) {
-  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    if (DT == KVB_DT_BF16) {
-      f[2 * i] = __uint_as_float(w[i] << 16);
-      f[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-    } else {
-      const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&w[i]));
-      f[2 * i] = t.x;
-      f[2 * i + 1] = t.y;
-    }
-  }
+__device__ __forceinline__ uint64_t unpack_pair(uint32_t w) {
+  if (DT == KVB_DT_BF16) return f2_pack(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+  const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&w));
+  return f2_pack(t.x, t.y);
 }
 
+// ||a-b||^2, ||a||^2, ||b||^2 over this lane's 8 elements, in packed float32 pairs
 template <int DT>
 __device__ __forceinline__ void row_sums(const uint4& a, const uint4& b, float& d2, float& na2, float& nb2) {
-  float x[8], y[8];
-  unpack8<DT>(a, x);
-  unpack8<DT>(b, y);
-  d2 = na2 = nb2 = 0.f;
+  const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+  uint64_t sd = 0ull, sa = 0ull, sb = 0ull;  // bit pattern of (+0, +0)
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const float df = x[i] - y[i];
-    d2 = fmaf(df, df, d2);
-    na2 = fmaf(x[i], x[i], na2);
-    nb2 = fmaf(y[i], y[i], nb2);
+  for (int i = 0; i < 4; ++i) {
+    const uint64_t x = unpack_pair<DT>(aw[i]), y = unpack_pair<DT>(bw[i]);
+    const uint64_t df = f2_sub(x, y);
+    sd = f2_fma(df, df, sd);
+    sa = f2_fma(x, x, sa);
+    sb = f2_fma(y, y, sb);
   }
+  d2 = f2_hsum(sd);
+  na2 = f2_hsum(sa);
+  nb2 = f2_hsum(sb);
 }
 
 __device__ __forceinline__ float one_minus_cos(float d2, float na2, float nb2) {
@@ -89,6 +85,7 @@ __global__ void __launch_bounds__(kThreads)
   const int n_hw = (kThreads / 32) * 2;
   const bool pair_same_token = (H % 2) == 0;  // rows u, u+1 (u even) belong to one token
 
+#pragma unroll 2
   for (int u0 = u_begin + warp * 2; u0 < u_end; u0 += n_hw) {
     const int u = u0 + s;
     const bool live = u < u_end;

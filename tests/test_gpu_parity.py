@@ -146,9 +146,11 @@ def test_assemble_all_modes_and_shifts(Hkv, Hq, kv_dtype):
         check_assembled(sh, r, g, exact, kv_o)
         # chunks 0, 1, 2 keep their position: rotation is the identity, unquantised rows are bit copies
         assert np.array_equal(g[:, :, 256:384], np.stack([helpers.bits_of(r.chunks_host[2].k_codes), helpers.bits_of(r.chunks_host[2].v_codes)], 1))
-        # values are never rotated: dequantisation alone, whatever the shift (float32 then 16-bit
-        # rounding on the GPU against one rounding from double: a stray last-bit difference at most)
-        assert np.mean(g[:, 1] == kv_o[:, 1]) > 0.9999
+        # values are never rotated: dequantisation alone, whatever the shift.  The GPU rounds a float32
+        # result (error <= 3 * 2^-24 relative) to 16 bits, the oracle rounds the exact value once: they
+        # differ only when the value sits that close to a rounding boundary (spacing 2^-11 relative in
+        # fp16), i.e. for at most 2 * 3 * 2^-24 / 2^-11 = 7e-4 of the values
+        assert np.mean(g[:, 1] == kv_o[:, 1]) > 0.9993
     finally:
         B.kvb_destroy(ctx)
 
