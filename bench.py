@@ -234,6 +234,20 @@ def run_reference(args, wl):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------------------- multi-rank glue
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of device-measured times over all ranks (the slowest rank sets
+    the job's time).  The path itself never communicates: ranks are independent replicas."""
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def job_throughput(world: int, tokens_per_rank_step: int, ms_per_step: float) -> float:
+    """Whole-job tokens/s: every rank processes its own batch per step (weak scaling)."""
+    return world * tokens_per_rank_step / (ms_per_step * 1e-3)
+
+
 # --------------------------------------------------------------------------------------- main arm
 def main():
     ap = argparse.ArgumentParser()
@@ -243,11 +257,14 @@ def main():
     ap.add_argument("--impl", default="kvb", choices=["kvb", "reference"])
     ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOADS))
     ap.add_argument("--replicas", type=int, default=0, help="independent copies rotated through (0 = auto)")
+    ap.add_argument("--batch", type=int, default=1, help="requests per step: the workload's request list repeated this many times")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     wl = synth.workload(WORKLOADS[args.workload])
+    if args.batch > 1:
+        wl = synth.Workload("%s_x%d" % (wl.name, args.batch), wl.seed, wl.shape, wl.requests * args.batch, wl.select, wl.sigma_bulk, wl.sigma_seam, wl.seam_tokens)
     if args.impl == "reference":
         run_reference(args, wl)
         return
@@ -359,15 +376,14 @@ def main():
     attn_flops = float(np.mean(flops))
 
     if dist:
-        t = torch.tensor([ms_total] + stage_ms + ([e2e["ms_per_step"]] if e2e else [0.0]), device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, stage_ms = float(t[0]), [float(x) for x in t[1:4]]
+        t = max_over_ranks([ms_total] + stage_ms + ([e2e["ms_per_step"]] if e2e else [0.0]), dist, dev)
+        ms_total, stage_ms = t[0], t[1:4]
         if e2e:
-            e2e["ms_per_step"] = float(t[4])
+            e2e["ms_per_step"] = t[4]
 
     peaks = load_peaks()
     ms_step = ms_total / args.steps
-    value = world * n_tok / (ms_step * 1e-3)
+    value = job_throughput(world, n_tok, ms_step)
     long_run = ms_total > 1000.0
     tensor_peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
     stages = {
@@ -396,7 +412,7 @@ def main():
         "clocks": sampler.summary(), "wall_s_timed": t_wall,
     }
     if e2e:
-        line["e2e"] = {"value": world * n_tok / (e2e["ms_per_step"] * 1e-3), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
+        line["e2e"] = {"value": job_throughput(world, n_tok, e2e["ms_per_step"]), "unit": UNIT, "h2d_bytes_per_step": e2e["h2d"],
                        "d2h_bytes_per_step": e2e["d2h"], "ms_per_step": e2e["ms_per_step"], "steps": e2e["steps"]}
 
     # ---- CPU oracle beside it (rank 0, N=1 only): bounded sample of the same workload
