@@ -395,7 +395,14 @@ def main():
         s["frac"] = s["achieved"] / s["peak"]
     top = max(stages, key=lambda k: stages[k]["ms"])
     roof = {k: stages[top][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
-    roof.update({"kernel": top, "traffic": None, "peak_source": "%s (%s)" % (peaks["source"], "sustained" if (top == "selective_attn" and long_run) else "burst/copy"),
+    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed ncu captures
+    # (profiles/cfg1_launches_and_kernels.md, profiles/cfg2_kernels.md); null where none was taken
+    ncu_traffic = {
+        ("cfg1_qwen3b_2k_int8", "selective_attn"): 207.0e6, ("cfg1_qwen3b_2k_int8", "assemble"): 67.6e6,
+        ("cfg1_qwen3b_2k_int8", "deviation_topk"): 154.2e6, ("cfg2_long_int4_8k", "selective_attn"): 647.1e6,
+        ("cfg2_long_int4_8k", "assemble"): 381.0e6, ("cfg2_long_int4_8k", "deviation_topk"): 608.2e6,
+    }
+    roof.update({"kernel": top, "traffic": ncu_traffic.get((wl.name, top)), "peak_source": "%s (%s)" % (peaks["source"], "sustained" if (top == "selective_attn" and long_run) else "burst/copy"),
                  "timing": "CUDA events around the C-ABI call of the stage, averaged over the timed steps"})
 
     line = {
@@ -417,12 +424,14 @@ def main():
 
     # ---- CPU oracle beside it (rank 0, N=1 only): bounded sample of the same workload
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        reqs_host = host_copy(reps[0].reqs)
-        n_l = 2 if n_tok <= 4096 else 1
-        if n_tok > 20000:  # ragged batch: the two shortest requests only
-            order = sorted(range(len(reqs_host)), key=lambda i: reqs_host[i].plan.T)[:2]
-            reqs_host = [reqs_host[i] for i in order]
-        secs, threads = oracle_sample_seconds(wl, reqs_host, n_l)
+        order = sorted(range(len(reps[0].reqs)), key=lambda i: reps[0].reqs[i].plan.T)
+        if n_tok > 20000:  # a batch: the four shortest requests only
+            order = order[:4]
+        reqs_host = host_copy([reps[0].reqs[i] for i in order])
+        # one layer first to calibrate, then as many layers as make about 12 s of CPU work
+        t1, threads = oracle_sample_seconds(wl, reqs_host, 1)
+        n_l = max(1, min(sh.L, int(round(12.0 / max(t1, 1e-3)))))
+        secs = t1 if n_l == 1 else oracle_sample_seconds(wl, reqs_host, n_l)[0]
         tok_s = sum(r.plan.T for r in reqs_host)
         line["cpu_baseline"] = {
             "value": tok_s / (secs * sh.L / n_l), "unit": UNIT, "cores": threads, "kind": "oracle",
