@@ -162,6 +162,21 @@ int kvb_deviation_topk(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const k
 int kvb_selective_attn(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_selection* sel,
                        const void* const* q, void* const* out, float softmax_scale, void* cuda_stream);
 
+/* CacheBlendRecompute (Algorithm 2) step 4, which is also the splice of
+ * SelectiveRecompute (Algorithm 1): for every request and every i < *n_sel,
+ * the K and V rows of position sel[i] in every layer of kv_buf are replaced
+ * by the rows of `fresh` (K~, V~).  sel: host array of n_req kvb_selection
+ * (only sel, n_sel, sel_capacity are read).  Other rows are not touched. */
+int kvb_patch(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_selection* sel, void* cuda_stream);
+
+/* Importance score of the cache manager's eviction policy (KV Cache Manager,
+ * Eq. 7): importance[r][c] = 1/(L*H*C) * sum over layers, KV heads and the C
+ * tokens of chunk c of ||k||_2, read from the stitched kv_buf (a rotation
+ * leaves the norms unchanged).  importance: host array of n_req device
+ * pointers, each to n_chunks float32 values. */
+int kvb_chunk_importance(kvb_ctx* ctx, const kvb_request* reqs, int n_req, float* const* importance,
+                         void* cuda_stream);
+
 /* KV Quantization, Eq. 6 (cache-population side), for one chunk: x [L][C][H][d]
  * in kv_dtype (device) -> codes and (scale, min) metadata in the layouts above.
  * is_value = 0: keys, per channel; 1: values, per token.  bits: 4 or 8. */

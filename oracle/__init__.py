@@ -217,3 +217,23 @@ def attention(q, kv_buf, sel, Hq: int, dtype: int, scale: float, layers=None, ro
         _p(layers), int(layers.size), _p(rows_a), 0 if rows_a is None else int(rows_a.size), _p(out), _p(exact),
     )
     return (out, exact) if want_exact else out
+
+
+# ---------------------------------------------------------------- Algorithm 2 step 4; Eq. 7
+def patch(kv_buf, fresh, sel) -> np.ndarray:
+    """Copy of kv_buf with the rows of the selected positions replaced by the fresh ones."""
+    kv = np.array(kv_buf, dtype=np.uint16, order="C", copy=True)
+    fresh = _c(fresh, np.uint16)
+    sel = _c(sel, np.int32)
+    L, _, T, H, d = kv.shape
+    lib().kvo_patch(_p(kv), _p(fresh), _p(sel), int(sel.size), L, T, H, d)
+    return kv
+
+
+def importance(kv_buf, C_tokens: int, dtype: int) -> np.ndarray:
+    """Mean key norm of every chunk of a stitched buffer (Eq. 7)."""
+    kv = _c(kv_buf, np.uint16)
+    L, _, T, H, d = kv.shape
+    out = np.empty(T // C_tokens, np.float64)
+    lib().kvo_importance(_p(kv), L, T, H, d, C_tokens, dtype, _p(out))
+    return out

@@ -24,6 +24,8 @@
  *                                     united with the top-k set
  *   kvo_attention                     Eq. 2 (causal softmax attention) for the
  *                                     selected query rows, GQA head mapping
+ *   kvo_patch                         Algorithm 2 step 4 / Algorithm 1 splice
+ *   kvo_importance                    Eq. 7 (mean key norm of a chunk)
  *
  * Pins (tests/test_oracle_*.py): every function above is pinned to closed
  * forms, invariants, brute force or a library routine; the three format
@@ -502,4 +504,45 @@ int kvo_max_threads(void) {
 #else
   return 1;
 #endif
+}
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 2, step 4 (and Algorithm 1's splice): patch                */
+/* ------------------------------------------------------------------ */
+
+/* Replaces the K and V rows of every selected position, in every layer, by the
+ * freshly projected ones:  KV[l, :, sel[i], :, :] <- fresh[l, :, sel[i], :, :]. */
+void kvo_patch(uint16_t* kv_buf, const uint16_t* fresh, const int32_t* sel, int n_sel, int L, int T, int H, int d) {
+  int64_t row = (int64_t)H * d;
+  for (int l = 0; l < L; l++)
+    for (int kv = 0; kv < 2; kv++)
+      for (int i = 0; i < n_sel; i++) {
+        int64_t off = (((int64_t)l * 2 + kv) * T + sel[i]) * row;
+        memcpy(kv_buf + off, fresh + off, (size_t)row * 2);
+      }
+}
+
+/* ------------------------------------------------------------------ */
+/* Eq. 7: importance of a chunk = mean L2 norm of its keys              */
+/* ------------------------------------------------------------------ */
+
+/* importance[c] = 1/(L*H*C) * sum over layers, heads and the chunk's C tokens of ||k||_2,
+ * for the chunks [c*C, (c+1)*C) of a [L][2][T][H][d] buffer. */
+void kvo_importance(const uint16_t* kv_buf, int L, int T, int H, int d, int C, int dtype, double* importance) {
+  int n_chunks = T / C;
+  for (int c = 0; c < n_chunks; c++) {
+    double sum = 0;
+    for (int l = 0; l < L; l++)
+      for (int t = c * C; t < (c + 1) * C; t++)
+        for (int h = 0; h < H; h++) {
+          const uint16_t* k = kv_buf + ((((int64_t)l * 2 + 0) * T + t) * H + h) * d;
+          double n2 = 0;
+          for (int j = 0; j < d; j++) {
+            double x = load16(k + j, dtype);
+            n2 += x * x;
+          }
+          sum += sqrt(n2);
+        }
+    importance[c] = sum / ((double)L * H * C);
+  }
 }

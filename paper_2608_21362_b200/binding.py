@@ -236,6 +236,21 @@ def kvb_selective_attn(ctx, table: RequestTable, sel: SelectionTable, q: List[to
     return _check(ctx, st) if check else st
 
 
+def kvb_patch(ctx, table: RequestTable, sel: SelectionTable, stream=None, check: bool = True) -> int:
+    L = lib()
+    L.kvb_patch.argtypes = [C.c_void_p, C.POINTER(kvb_request), C.c_int, C.POINTER(kvb_selection), C.c_void_p]
+    st = L.kvb_patch(ctx, table.array, table.n, sel.array, _stream(stream))
+    return _check(ctx, st) if check else st
+
+
+def kvb_chunk_importance(ctx, table: RequestTable, importance: List[torch.Tensor], stream=None, check: bool = True) -> int:
+    L = lib()
+    L.kvb_chunk_importance.argtypes = [C.c_void_p, C.POINTER(kvb_request), C.c_int, C.POINTER(C.c_void_p), C.c_void_p]
+    ptrs = (C.c_void_p * max(table.n, 1))(*[t.data_ptr() for t in importance])
+    st = L.kvb_chunk_importance(ctx, table.array, table.n, ptrs, _stream(stream))
+    return _check(ctx, st) if check else st
+
+
 def kvb_quantize_chunk(ctx, x: torch.Tensor, is_value: bool, bits: int, codes: torch.Tensor, meta: torch.Tensor,
                        stream=None, check: bool = True) -> int:
     st = lib().kvb_quantize_chunk(ctx, x.data_ptr(), int(is_value), bits, codes.data_ptr(), meta.data_ptr(), _stream(stream))

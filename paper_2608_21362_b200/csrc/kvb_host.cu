@@ -436,6 +436,77 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
   return KVB_OK;
 }
 
+int kvb_patch(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_selection* sel, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  if (!sel) return fail(c, KVB_ERR_INVALID_ARG, "NULL selection array");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
+  const int rows_per_cta = 64;
+  int tiles = 0;
+  for (int r = 0; r < n_req; ++r) {
+    const kvb_selection& s = sel[r];
+    if (!s.sel || !s.n_sel || s.sel_capacity <= 0) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL sel / n_sel or empty capacity", r);
+    ReqDesc d{};
+    d.kv_buf = static_cast<const uint8_t*>(reqs[r].kv_buf);
+    d.fresh = static_cast<const uint8_t*>(reqs[r].fresh);
+    d.sel = s.sel;
+    d.n_sel = s.n_sel;
+    d.T = reqs[r].T;
+    d.sel_capacity = s.sel_capacity;
+    d.tile_offset = tiles;
+    rd[r] = d;
+    tiles += (s.sel_capacity + rows_per_cta - 1) / rows_per_cta;
+  }
+  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  KVB_CUDA(c, launch_patch(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, tiles, rows_per_cta, c->dims, st));
+  c->launches += 1;
+  return KVB_OK;
+}
+
+int kvb_chunk_importance(kvb_ctx* c, const kvb_request* reqs, int n_req, float* const* importance, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  if (!importance) return fail(c, KVB_ERR_INVALID_ARG, "NULL importance array");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
+  int chunks = 0;
+  for (int r = 0; r < n_req; ++r) {
+    if (!importance[r]) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL importance output", r);
+    ReqDesc d{};
+    d.kv_buf = static_cast<const uint8_t*>(reqs[r].kv_buf);
+    d.delta = importance[r];  // the descriptor's float output slot
+    d.T = reqs[r].T;
+    d.tile_offset = chunks;
+    rd[r] = d;
+    chunks += reqs[r].n_chunks;
+  }
+  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  KVB_CUDA(c, launch_importance(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, chunks, c->dims, st));
+  c->launches += 1;
+  return KVB_OK;
+}
+
 int kvb_quantize_chunk(kvb_ctx* c, const void* x, int is_value, int bits, void* codes, void* meta, void* cuda_stream) {
   if (!c) return KVB_ERR_INVALID_ARG;
   if (!x || !codes || !meta || (bits != 4 && bits != 8)) return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");

@@ -85,6 +85,10 @@ int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity
 cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,
                                 float scale, uint32_t* status, cudaStream_t st);
 
+cudaError_t launch_patch(const ReqDesc* reqs, int n_req, int total_tiles, int rows_per_cta, const ModelDims& m,
+                         cudaStream_t st);
+cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, cudaStream_t st);
+
 cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
                             cudaStream_t st);
 

@@ -420,3 +420,38 @@ def test_golden_fixture_rope_worked_example():
     for j, (ang, c, s) in enumerate(rows):
         assert R[j, j] == pytest.approx(c, abs=1e-12) and R[j + 4, j] == pytest.approx(s, abs=1e-12)
         assert R[j, j + 4] == pytest.approx(-s, abs=1e-12) and R[j + 4, j + 4] == pytest.approx(c, abs=1e-12)
+
+
+# ------------------------------------------------------------------ Algorithm 2 step 4; Eq. 7
+def test_patch_replaces_exactly_the_selected_rows():
+    L, T, H, d = 3, 20, 2, 8
+    kv = _rand_bits((L, 2, T, H, d), 1)
+    fresh = _rand_bits((L, 2, T, H, d), 1)
+    sel = np.array([0, 3, 4, 19], np.int32)
+    got = oracle.patch(kv, fresh, sel)
+    want = kv.copy()
+    want[:, :, sel] = fresh[:, :, sel]  # numpy indexed assignment as the plain definition
+    assert np.array_equal(got, want)
+    assert np.array_equal(oracle.patch(kv, fresh, np.zeros(0, np.int32)), kv)
+    # a patched position no longer deviates; the others keep their deviation
+    d_before = oracle.deviation(kv, fresh, 1, 3)[0]
+    d_after = oracle.deviation(got, fresh, 1, 3)[0]
+    assert np.all(d_after[sel] == 0.0)
+    rest = np.setdiff1d(np.arange(T), sel)
+    assert np.array_equal(d_after[rest], d_before[rest])
+
+
+def test_importance_is_the_mean_key_norm():
+    L, T, H, d, C = 2, 12, 2, 16, 4
+    kv = _rand_bits((L, 2, T, H, d), 1)
+    K = oracle.bits_to_f64(kv[:, 0], 1)  # [L,T,H,d]
+    want = np.linalg.norm(K, axis=-1).reshape(L, T // C, C, H).mean(axis=(0, 2, 3))
+    assert np.allclose(oracle.importance(kv, C, 1), want, rtol=0, atol=1e-14)
+    # closed forms: all-ones keys have norm sqrt(d); values never matter; scaling is linear
+    ones = oracle.round_to_bits(np.ones((L, 2, T, H, d)), 1)
+    assert np.allclose(oracle.importance(ones, C, 1), math.sqrt(d), atol=1e-15)
+    kv2 = kv.copy()
+    kv2[:, 1] = ones[:, 1]
+    assert np.array_equal(oracle.importance(kv2, C, 1), oracle.importance(kv, C, 1))
+    dbl = oracle.round_to_bits(oracle.bits_to_f64(kv, 1) * 2.0, 1)
+    assert np.allclose(oracle.importance(dbl, C, 1), 2 * oracle.importance(kv, C, 1), rtol=1e-15)
