@@ -31,10 +31,11 @@ void* g_scratch_addr[kMaxDevices] = {nullptr};
 
 __global__ void store_desc_kernel(ReqDesc d, ReqDesc* dst) { *dst = d; }
 
-__global__ void finalize_delta_kernel(const unsigned long long* __restrict__ acc, int T, double inv_terms,
+// same arithmetic as the selection kernel of the context path: one conversion, one multiplication
+__global__ void finalize_delta_kernel(const unsigned long long* __restrict__ acc, int T, float inv_scale,
                                       float* __restrict__ delta) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t < T) delta[t] = (float)((double)(long long)acc[t] * (1.0 / 1099511627776.0) * inv_terms);
+  if (t < T) delta[t] = __ll2float_rn((long long)acc[t]) * inv_scale;
 }
 
 }  // namespace
@@ -75,7 +76,7 @@ extern "C" int kvb_deviation_static(int device, const kvb_model_desc* model, con
   const int tiles = (T + deviation_tile_tokens() - 1) / deviation_tile_tokens();
   if (launch_deviation(desc_dev, 1, tiles, dims, which, acc, st) != cudaSuccess) return KVB_ERR_CUDA;
   const int n_terms = m.L * m.Hkv * ((which & 1) + ((which >> 1) & 1));
-  finalize_delta_kernel<<<(T + 255) / 256, 256, 0, st>>>(acc, T, 1.0 / (double)n_terms, delta);
+  finalize_delta_kernel<<<(T + 255) / 256, 256, 0, st>>>(acc, T, (float)(1.0 / (1099511627776.0 * (double)n_terms)), delta);
   if (cudaGetLastError() != cudaSuccess) return KVB_ERR_CUDA;
   return KVB_OK;
 }

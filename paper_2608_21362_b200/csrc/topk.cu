@@ -6,13 +6,16 @@
 //   3. bitonic sort of the k (key, index) pairs -> rank, most deviated first;
 //   4. bitmask union with the seam windows, prefix sum -> ascending sel and n_sel.
 // All decisions are integer comparisons: the result is a pure function of the float32 delta.
+// The kernel is latency-bound (one CTA, at most 128 KB of keys), so it is written to need few
+// block-wide barriers: warp-aggregated histogram updates, one combined prefix sum for the
+// selection, conflict-free shared-memory access, and the bitonic stages with stride < 32 done
+// in registers with shuffles.
 #include "kvb_internal.h"
 
 namespace kvb {
 namespace {
 
 constexpr int kThreads = 1024;
-constexpr int kWarps = kThreads / 32;
 constexpr int kMaxT = 32768;  // one 32-bit mask word per thread
 constexpr int kMaxK = 8192;
 
@@ -53,57 +56,72 @@ __device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* w
   return res;
 }
 
+__device__ __forceinline__ unsigned long long shfl_xor64(unsigned long long v, int o) {
+  return __shfl_xor_sync(0xffffffffu, v, o);
+}
+// one compare-exchange step of a bitonic network held one element per lane
+__device__ __forceinline__ unsigned long long ce_step(unsigned long long v, int lane, int stride, bool up) {
+  const unsigned long long o = shfl_xor64(v, stride);
+  const bool take_min = ((lane & stride) == 0) == up;
+  return take_min ? (v < o ? v : o) : (v > o ? v : o);
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-    topk_kernel(const ReqDesc* __restrict__ reqs, const SeamWindow* __restrict__ seams, double inv_terms,
+    topk_kernel(const ReqDesc* __restrict__ reqs, const SeamWindow* __restrict__ seams, float inv_scale,
                 unsigned long long* __restrict__ acc, int t_pad, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
-  uint32_t* s_keys = reinterpret_cast<uint32_t*>(smem);                           // [t_pad]
-  uint32_t* s_mask = s_keys + t_pad;                                              // [kThreads] selection bitmask
-  unsigned long long* s_comp = reinterpret_cast<unsigned long long*>(s_mask + kThreads);  // [k_pad] / histograms
-  uint32_t* s_hist = reinterpret_cast<uint32_t*>(s_comp);                         // [kWarps][256], aliases s_comp
+  uint32_t* s_keys = reinterpret_cast<uint32_t*>(smem);                                   // [t_pad]
+  uint32_t* s_mask = s_keys + t_pad;                                                      // [kThreads] selection bitmask
+  unsigned long long* s_comp = reinterpret_cast<unsigned long long*>(s_mask + kThreads);  // [k_pad]
   __shared__ uint32_t s_warp_sums[33];
-  __shared__ uint32_t s_bins[256];
-  __shared__ uint32_t s_sel[2];  // chosen bin, remaining need
+  __shared__ uint32_t s_hist[2][256];  // two buffers: one is cleared while the other is scanned
+  __shared__ uint32_t s_pick[2];       // chosen bin, remaining need
 
   const ReqDesc rq = reqs[blockIdx.x];
   const int T = rq.T, k = min(rq.k, T);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  // ---- 1. delta and keys
+  // ---- 1. delta and keys.  The sums are integers below 2^50 (units of 2^-40); one conversion to
+  //      float32 and one multiplication by 2^-40 / n_terms give delta to 1.2e-7 relative.
   for (int t = tid; t < T; t += kThreads) {
     const unsigned long long a = acc[rq.tok_offset + t];
     acc[rq.tok_offset + t] = 0ull;
-    const float dl = (float)((double)(long long)a * (1.0 / 1099511627776.0) * inv_terms);
+    const float dl = __ll2float_rn((long long)a) * inv_scale;
     rq.delta[t] = dl;
     s_keys[t] = order_key(dl);
   }
-  s_mask[tid] = 0u;
+  if (tid < 256) s_hist[1][tid] = 0u;  // the first pass (pass 3) counts into buffer 1
   __syncthreads();
 
   // ---- 2. radix select: threshold key `prefix`, and how many keys equal to it are taken (`need`)
   uint32_t prefix = 0, mask = 0, need = (uint32_t)k;
   if (k > 0 && k < T) {
     for (int pass = 3; pass >= 0; --pass) {
-      for (int i = tid; i < kWarps * 256; i += kThreads) s_hist[i] = 0;
-      __syncthreads();
+      uint32_t* hist = s_hist[pass & 1];
       const int shift = pass * 8;
-      for (int t = tid; t < T; t += kThreads) {
-        const uint32_t key = s_keys[t];
-        if ((key & mask) == prefix) atomicAdd(&s_hist[warp * 256 + ((key >> shift) & 255u)], 1u);
+      for (int t0 = 0; t0 < T; t0 += kThreads) {  // whole warps stay together for the votes
+        const int t = t0 + tid;
+        const uint32_t key = t < T ? s_keys[t] : 0u;
+        const bool in = t < T && (key & mask) == prefix;
+        const uint32_t digit = (key >> shift) & 255u;
+        const uint32_t members = __ballot_sync(0xffffffffu, in);
+        if (members == 0u) continue;
+        const int leader = __ffs(members) - 1;
+        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, leader);
+        if (__all_sync(0xffffffffu, !in || digit == d0)) {  // the high digits of nearby deviations mostly agree
+          if (lane == leader) atomicAdd(&hist[d0], (uint32_t)__popc(members));
+        } else if (in) {
+          atomicAdd(&hist[digit], 1u);
+        }
       }
-      __syncthreads();
-      if (tid < 256) {
-        uint32_t c = 0;
-        for (int w = 0; w < kWarps; ++w) c += s_hist[w * 256 + tid];
-        s_bins[tid] = c;
-      }
+      if (tid < 256) s_hist[(pass & 1) ^ 1][tid] = 0u;  // the next pass's histogram
       __syncthreads();
       if (warp == 0) {
         // lane j owns bins 255-8j .. 248-8j (descending); find the bin where the running count reaches need
         uint32_t local[8], sum = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          local[i] = s_bins[255 - (lane * 8 + i)];
+          local[i] = hist[255 - (lane * 8 + i)];
           sum += local[i];
         }
         uint32_t inc = sum;
@@ -117,30 +135,32 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             if (before < need && before + local[i] >= need) {
-              s_sel[0] = 255 - (lane * 8 + i);
-              s_sel[1] = need - before;
+              s_pick[0] = 255 - (lane * 8 + i);
+              s_pick[1] = need - before;
             }
             before += local[i];
           }
         }
       }
       __syncthreads();
-      prefix |= s_sel[0] << shift;
+      prefix |= s_pick[0] << shift;
       mask |= 255u << shift;
-      need = s_sel[1];
-      __syncthreads();
+      need = s_pick[1];
     }
   }
 
-  // ---- 3. the top-k set in index order; thread w owns positions 32w .. 32w+31
+  // ---- 3. the top-k set in index order; thread w owns positions 32w .. 32w+31 (read in a
+  //      lane-rotated order so that the 32 lanes of a warp hit 32 different banks)
   uint32_t gt_mask = 0, eq_mask = 0;
   {
     const int base = tid * 32;
     if (k >= T) {
       for (int i = 0; i < 32; ++i)
         if (base + i < T) gt_mask |= 1u << i;
-    } else if (k > 0) {
-      for (int i = 0; i < 32; ++i) {
+    } else if (k > 0 && base < T) {
+#pragma unroll 8
+      for (int j = 0; j < 32; ++j) {
+        const int i = (j + lane) & 31;
         if (base + i < T) {
           const uint32_t key = s_keys[base + i];
           if (key > prefix) gt_mask |= 1u << i;
@@ -149,52 +169,92 @@ __global__ void __launch_bounds__(kThreads, 1)
       }
     }
   }
-  uint32_t tot_eq, tot_sel;
-  const uint32_t eq_before = block_exclusive_scan(__popc(eq_mask), s_warp_sums, &tot_eq);
-  uint32_t sel_mask = gt_mask;
+  // one scan for both counts (each at most 32768: 16 bits apiece)
+  uint32_t tot_packed;
+  const uint32_t packed_before =
+      block_exclusive_scan((uint32_t)__popc(gt_mask) | ((uint32_t)__popc(eq_mask) << 16), s_warp_sums, &tot_packed);
+  const uint32_t gt_before = packed_before & 0xFFFFu, eq_before = packed_before >> 16;
+  const uint32_t n_take_eq = (k > 0 && k < T) ? need : 0u;  // threshold-valued keys taken, lowest indices first
+  int k_pad = 1;
+  while (k_pad < k) k_pad <<= 1;
+  // composite sort keys (larger delta first, then lower index) of the selected positions, in index order
   {
+    uint32_t sel_mask = gt_mask;
     uint32_t e = eq_mask, r = eq_before;
     while (e) {
       const int b = __ffs(e) - 1;
       e &= e - 1;
-      if (r < need && k < T) sel_mask |= 1u << b;
+      if (r < n_take_eq) sel_mask |= 1u << b;
       ++r;
     }
-  }
-  const uint32_t sel_before = block_exclusive_scan(__popc(sel_mask), s_warp_sums, &tot_sel);
-  int k_pad = 1;
-  while (k_pad < k) k_pad <<= 1;
-  // composite sort keys: larger delta first, then lower index
-  for (int i = tid; i < k_pad; i += kThreads) s_comp[i] = ~0ull;
-  __syncthreads();
-  {
-    uint32_t e = sel_mask, pos = sel_before;
-    while (e) {
-      const int b = __ffs(e) - 1;
-      e &= e - 1;
+    uint32_t pos = gt_before + min(eq_before, n_take_eq);
+    uint32_t m2 = sel_mask;
+    while (m2) {
+      const int b = __ffs(m2) - 1;
+      m2 &= m2 - 1;
       const uint32_t t = tid * 32 + b;
       if (pos < (uint32_t)k_pad) s_comp[pos] = ((unsigned long long)(~s_keys[t]) << 32) | t;
       ++pos;
     }
+    s_mask[tid] = sel_mask;
   }
-  s_mask[tid] = sel_mask;
+  for (int i = k + tid; i < k_pad; i += kThreads) s_comp[i] = ~0ull;  // padding sorts last
+  const uint32_t tot_sel = (tot_packed & 0xFFFFu) + min(tot_packed >> 16, n_take_eq);
   __syncthreads();
 
-  // ---- bitonic sort of s_comp[0..k_pad)
-  for (int size = 2; size <= k_pad; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int i = tid; i < (k_pad >> 1); i += kThreads) {
-        const int lo = 2 * i - (i & (stride - 1));
-        const int hi = lo + stride;
-        const bool up = (lo & size) == 0;
-        const unsigned long long a = s_comp[lo], b = s_comp[hi];
-        if ((a > b) == up) {
-          s_comp[lo] = b;
-          s_comp[hi] = a;
+  // ---- bitonic sort of s_comp[0..k_pad): element i lives in lane i % 32 of its warp for the steps
+  //      with stride < 32 (registers + shuffles); larger strides go through shared memory
+  if (k_pad >= 32) {
+    for (int i0 = 0; i0 < k_pad; i0 += kThreads) {  // sizes 2..32 entirely in registers
+      const int i = i0 + tid;
+      if (i0 + (tid & ~31) >= k_pad) break;  // whole warps only (k_pad is a multiple of 32)
+      unsigned long long v = s_comp[i];
+#pragma unroll
+      for (int size = 2; size <= 32; size <<= 1) {
+        const bool up = (i & size) == 0;
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+      }
+      s_comp[i] = v;
+    }
+    __syncthreads();
+    for (int size = 64; size <= k_pad; size <<= 1) {
+      for (int stride = size >> 1; stride >= 32; stride >>= 1) {
+        for (int i = tid; i < (k_pad >> 1); i += kThreads) {
+          const int lo = 2 * i - (i & (stride - 1));
+          const int hi = lo + stride;
+          const bool up = (lo & size) == 0;
+          const unsigned long long a = s_comp[lo], b = s_comp[hi];
+          if ((a > b) == up) {
+            s_comp[lo] = b;
+            s_comp[hi] = a;
+          }
         }
+        __syncthreads();
+      }
+      for (int i0 = 0; i0 < k_pad; i0 += kThreads) {  // strides 16..1 of this size
+        const int i = i0 + tid;
+        if (i0 + (tid & ~31) >= k_pad) break;
+        unsigned long long v = s_comp[i];
+        const bool up = (i & size) == 0;
+#pragma unroll
+        for (int stride = 16; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+        s_comp[i] = v;
       }
       __syncthreads();
     }
+  } else {
+    if (warp == 0) {  // fewer than 32 elements: one warp, padded with keys that sort last
+      unsigned long long v = lane < k_pad ? s_comp[lane] : ~0ull;
+#pragma unroll
+      for (int size = 2; size <= 32; size <<= 1) {
+        const bool up = (lane & size) == 0;
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+      }
+      if (lane < k_pad) s_comp[lane] = v;
+    }
+    __syncthreads();
   }
   for (int i = tid; i < k; i += kThreads) rq.rank[i] = (int32_t)(uint32_t)(s_comp[i] & 0xFFFFFFFFull);
 
@@ -231,11 +291,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 int topk_max_T() { return kMaxT; }
 int topk_max_k() { return kMaxK; }
 
-static size_t topk_smem(int t_pad, int k_pad) {
-  size_t comp = (size_t)k_pad * 8;
-  if (comp < (size_t)kWarps * 256 * 4) comp = (size_t)kWarps * 256 * 4;
-  return (size_t)t_pad * 4 + kThreads * 4 + comp;
-}
+static size_t topk_smem(int t_pad, int k_pad) { return (size_t)t_pad * 4 + kThreads * 4 + (size_t)(k_pad < 32 ? 32 : k_pad) * 8; }
 
 cudaError_t topk_configure() {
   return cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -248,7 +304,8 @@ cudaError_t launch_topk(const ReqDesc* reqs, int n_req, const SeamWindow* seams,
   int t_pad = (max_T + 31) & ~31;
   int k_pad = 1;
   while (k_pad < max_k) k_pad <<= 1;
-  topk_kernel<<<n_req, kThreads, topk_smem(t_pad, k_pad), st>>>(reqs, seams, 1.0 / (double)n_terms, acc, t_pad, status);
+  const float inv_scale = (float)(1.0 / (1099511627776.0 * (double)n_terms));  // 2^-40 / n_terms
+  topk_kernel<<<n_req, kThreads, topk_smem(t_pad, k_pad), st>>>(reqs, seams, inv_scale, acc, t_pad, status);
   return cudaGetLastError();
 }
 
