@@ -249,9 +249,16 @@ __global__ void __launch_bounds__(kThreads, 2)
   }
   const ReqDesc rq = reqs[lo];
   const int tiles_r = (rq.sel_capacity + TOK - 1) / TOK;
+  // Within a request: (layer, head) pairs go in groups of rq.lhk_group whose K/V planes fit L2
+  // together; inside a group the order is tile-major from the longest tile down (longest-first
+  // packing over the whole group), the pairs of the group interleaved.
   const int idx = lin - rq.tile_offset * per_tile;
-  const int lhk = idx / tiles_r;
-  const int tile = tiles_r - 1 - idx % tiles_r;
+  const int G = rq.lhk_group;
+  const int grp = idx / (G * tiles_r);
+  const int rem = idx - grp * G * tiles_r;
+  const int g_eff = min(G, per_tile - grp * G);
+  const int lhk = grp * G + rem % g_eff;
+  const int tile = tiles_r - 1 - rem / g_eff;
   const int hk = lhk % m.Hkv;
   const int l = lhk / m.Hkv;
   const CUtensorMap* map_q = maps + 2 * lo;

@@ -417,6 +417,14 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
     d.T = reqs[r].T;
     d.sel_capacity = s.sel_capacity;
     d.tile_offset = tiles;
+    {  // (layer, head) pairs whose K and V planes (T * d * 2 * 2 bytes each) fit in about 48 MB of L2 together
+      const int lh = c->model.L * c->model.Hkv;
+      const double pair_bytes = (double)reqs[r].T * c->model.d * 4.0;
+      int g0 = (int)(48.0e6 / pair_bytes);
+      g0 = g0 < 1 ? 1 : (g0 > lh ? lh : g0);
+      const int n_groups = (lh + g0 - 1) / g0;
+      d.lhk_group = (lh + n_groups - 1) / n_groups;
+    }
     rd[r] = d;
     tiles += (s.sel_capacity + tok_per_tile - 1) / tok_per_tile;
     if (!c->attn_legacy) {

@@ -46,7 +46,7 @@ struct ReqDesc {
   int32_t tile_offset;   // first tile of this request in a kernel's flat tile space
   int32_t seam_offset;   // first entry of this request in the seam window list
   int32_t n_seams;
-  int32_t pad;
+  int32_t lhk_group;     // attention: (layer, head) pairs per scheduling group
 };
 
 struct SeamWindow {
