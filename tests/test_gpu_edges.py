@@ -1,0 +1,129 @@
+"""Edge cases of the CUDA path: empty batches, the smallest and the largest requests the selection
+kernel takes, an empty selection, overlapping and clamped seam windows."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_21362_b200 import binding as B
+from paper_2608_21362_b200 import synth
+from paper_2608_21362_b200.build import build_library
+
+import helpers
+from test_gpu_parity import check_assembled, check_attention, check_selection, oracle_stitch, prepare, run_assemble, run_attention, run_select
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_library()
+
+
+def test_empty_batch_is_a_no_op():
+    sh = synth.Shape(L=2)
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        empty = B.RequestTable([])
+        sel = B.SelectionTable([], [], [], DEV)
+        assert B.kvb_assemble(ctx, empty) == B.KVB_OK
+        assert B.kvb_deviation_topk(ctx, empty, 0.15, -1, 16, 0, 3, sel) == B.KVB_OK
+        assert B.kvb_selective_attn(ctx, empty, sel, [], [], 0.1) == B.KVB_OK
+        assert B.kvb_patch(ctx, empty, sel) == B.KVB_OK
+        assert B.kvb_launch_count(ctx) == 0 and B.kvb_last_status(ctx) == B.KVB_OK
+    finally:
+        B.kvb_destroy(ctx)
+
+
+def test_single_fresh_chunk_request():
+    """T = 128, nothing cached: the buffer is a copy of the fresh tensor, every deviation is 0, the
+    selection is the first floor(0.15 * 128) = 19 positions, there is no seam."""
+    sh = synth.Shape(L=2)
+    wl = synth.Workload("one", 3, sh, [synth._request(128, sh.C, [synth.MODE_FRESH], [0])], synth.SelectPlan())
+    reqs = prepare(wl)
+    (r,) = reqs
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        assert torch.equal(r.kv_buf.view(torch.int16), r.fresh.view(torch.int16))
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, use_oracle_buffer=False)
+        assert ks == [19] and int(sel.n_sel[0]) == 19
+        assert np.all(sel.delta[0].cpu().numpy() == 0.0)
+        assert sel.rank[0].cpu().numpy().tolist() == list(range(19)) == sel.sel[0].cpu().numpy()[:19].tolist()
+        outs = run_attention(ctx, sh, reqs, tbl, sel)
+        check_attention(sh, r, np.arange(19, dtype=np.int32), outs[0], None, None)
+    finally:
+        B.kvb_destroy(ctx)
+
+
+def test_selection_at_its_size_limits():
+    """T = 32768 with k = 8192 is the largest request the selection kernel takes; one more chunk or
+    one more selected position is refused before anything is launched."""
+    sh = synth.Shape(L=1)
+    n_chunks = 256
+    rng = np.random.default_rng(8)
+    modes = [synth.MODE_INT8 if rng.random() < 0.8 else synth.MODE_FRESH for _ in range(n_chunks)]
+    origs = (rng.permutation(1024)[:n_chunks] * sh.C).tolist()
+    sp = synth.SelectPlan(k_override=8192, seam_before=16, seam_after=0)
+    wl = synth.Workload("big", 8, sh, [synth._request(n_chunks * sh.C, sh.C, modes, origs)], sp)
+    reqs = prepare(wl)
+    ctx = B.create_for_shape(sh, 0, max_requests=1, max_chunks_total=n_chunks + 1, max_tokens_total=(n_chunks + 1) * sh.C)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, sp, use_oracle_buffer=False)
+        check_selection(sh, reqs, sel, ks, sp)
+        before = B.kvb_launch_count(ctx)
+        sel2 = B.SelectionTable([32768], [8193], [32768], DEV)
+        assert B.kvb_deviation_topk(ctx, tbl, 0.0, 8193, 0, 0, 3, sel2, check=False) == B.KVB_ERR_UNSUPPORTED
+        assert B.kvb_launch_count(ctx) == before
+    finally:
+        B.kvb_destroy(ctx)
+    # one chunk more than the kernel takes
+    wl2 = synth.Workload("too_big", 9, sh, [synth._request((n_chunks + 1) * sh.C, sh.C, [synth.MODE_FRESH] * (n_chunks + 1), [0] * (n_chunks + 1))], sp)
+    plan = wl2.requests[0]
+
+    class R:
+        pass
+
+    r = R()
+    r.plan, r.chunks = plan, [synth.Chunk(c) for c in plan.chunks]
+    r.kv_buf = torch.zeros((1, 2, plan.T, sh.Hkv, sh.d), dtype=torch.bfloat16, device=DEV)
+    r.fresh = torch.zeros_like(r.kv_buf)
+    ctx = B.create_for_shape(sh, 0, max_requests=1, max_chunks_total=n_chunks + 1, max_tokens_total=plan.T)
+    try:
+        sel3 = B.SelectionTable([plan.T], [10], [plan.T], DEV)
+        assert B.kvb_deviation_topk(ctx, B.RequestTable([r]), 0.0, 10, 0, 0, 3, sel3, check=False) == B.KVB_ERR_UNSUPPORTED
+        assert "limits" in B.kvb_last_error(ctx)
+    finally:
+        B.kvb_destroy(ctx)
+
+
+def test_empty_selection_and_wide_overlapping_seam_windows():
+    wl = synth.workload(0)
+    sh = wl.shape
+    reqs = prepare(wl)
+    (r,) = reqs
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        # nothing selected: k = 0 and no windows -> n_sel = 0, attention and patch touch nothing
+        sp0 = synth.SelectPlan(k_override=0, seam_before=0, seam_after=0)
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, sp0, use_oracle_buffer=False)
+        assert int(sel.n_sel[0]) == 0
+        sel_for_attn = B.SelectionTable([r.plan.T], [0], [r.sel_capacity], DEV)  # capacity of the Q tensor, n_sel = 0
+        out = torch.full_like(r.q, 3.0)
+        B.kvb_selective_attn(ctx, tbl, sel_for_attn, [r.q], [out], 0.1)
+        before = r.kv_buf.clone()
+        B.kvb_patch(ctx, tbl, sel_for_attn)
+        B.kvb_last_status(ctx)
+        assert torch.all(out == 3.0) and torch.equal(before.view(torch.int16), r.kv_buf.view(torch.int16))
+        # windows wider than a chunk: they overlap each other and are clamped at 0 and T
+        sp = synth.SelectPlan(ratio=0.05, seam_before=200, seam_after=150)
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, sp, use_oracle_buffer=False)
+        check_selection(sh, reqs, sel, ks, sp)
+        assert int(sel.n_sel[0]) == r.plan.T  # three seams x 350 positions cover all 512
+    finally:
+        B.kvb_destroy(ctx)

@@ -197,7 +197,7 @@ def run_select(ctx, wl, reqs, tbl, sp=None, use_oracle_buffer=True):
             r.kv_buf.copy_(r.kv_oracle.to(DEV))
     Ts = [r.plan.T for r in reqs]
     ks = [sp.k_override if sp.k_override >= 0 else B.kvb_select_count(T, sp.ratio) for T in Ts]
-    caps = [min(r.plan.T, k + (len(r.chunks) - 1) * (sp.seam_before + sp.seam_after)) for r, k in zip(reqs, ks)]
+    caps = [max(1, min(r.plan.T, k + (len(r.chunks) - 1) * (sp.seam_before + sp.seam_after))) for r, k in zip(reqs, ks)]
     sel = B.SelectionTable(Ts, ks, caps, DEV)
     B.kvb_deviation_topk(ctx, tbl, sp.ratio, sp.k_override, sp.seam_before, sp.seam_after, sp.which, sel)
     B.kvb_last_status(ctx)
