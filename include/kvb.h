@@ -118,6 +118,9 @@ typedef struct {
   int32_t seam_before; /* R of Algorithm 1: window [p-before, p+after) around each seam p */
   int32_t seam_after;
   int32_t which;       /* bit 0: keys (the printed deviation formula); bit 1: values */
+  int32_t sink_tokens; /* attention-sink tokens (Tokenization and Chunking): the first s positions of the
+                          prompt are always selected; 0 = off */
+  int32_t reserved;
 } kvb_select_params;
 
 /* Per-request outputs of the selection (device memory, caller-owned). */

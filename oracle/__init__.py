@@ -190,12 +190,12 @@ def topk(delta32, k: int) -> np.ndarray:
     return rank
 
 
-def seam_select(rank, chunk_new_pos, chunk_mode, T: int, before: int, after: int) -> np.ndarray:
+def seam_select(rank, chunk_new_pos, chunk_mode, T: int, before: int, after: int, sinks: int = 0) -> np.ndarray:
     rank = _c(rank, np.int32)
     pos = _c(chunk_new_pos, np.int32)
     mode = _c(chunk_mode, np.int32)
     sel = np.empty(max(T, 1), np.int32)
-    n = lib().kvo_seam_select(_p(rank), int(rank.size), _p(pos), _p(mode), int(pos.size), T, before, after, _p(sel))
+    n = lib().kvo_seam_select(_p(rank), int(rank.size), _p(pos), _p(mode), int(pos.size), T, before, after, int(sinks), _p(sel))
     return sel[:n].copy()
 
 

@@ -419,12 +419,15 @@ void kvo_topk(const float* delta, int T, int k, int32_t* rank) {
 /* A seam is an interior chunk boundary p = new_pos of chunk i >= 1 (chunks in
  * prompt order) where chunk i or chunk i-1 is cached (not FRESH).  Its window
  * is [max(0, p-before), min(T, p+after)); Algorithm 1 is (before, after) =
- * (R, 0).  sel = ascending, duplicate-free union of rank[0..k) and all
- * windows; returns n_sel.  sel must hold T entries. */
+ * (R, 0).  The first `sinks` positions (attention-sink tokens of the Tokenization
+ * and Chunking section) are always taken.  sel = ascending, duplicate-free
+ * union of rank[0..k), all windows and the sinks; returns n_sel.  sel must hold
+ * T entries. */
 int kvo_seam_select(const int32_t* rank, int k, const int32_t* chunk_new_pos, const int32_t* chunk_mode,
-                    int n_chunks, int T, int before, int after, int32_t* sel) {
+                    int n_chunks, int T, int before, int after, int sinks, int32_t* sel) {
   uint8_t* mark = (uint8_t*)calloc((size_t)(T > 0 ? T : 1), 1);
   for (int i = 0; i < k; i++) mark[rank[i]] = 1;
+  for (int t = 0; t < sinks && t < T; t++) mark[t] = 1;
   for (int c = 1; c < n_chunks; c++) {
     if (chunk_mode[c] == KVO_MODE_FRESH && chunk_mode[c - 1] == KVO_MODE_FRESH) continue;
     int p = chunk_new_pos[c];

@@ -65,7 +65,7 @@ class kvb_limits(C.Structure):
 class kvb_select_params(C.Structure):
     _fields_ = [
         ("ratio", C.c_double), ("k_override", C.c_int32), ("seam_before", C.c_int32),
-        ("seam_after", C.c_int32), ("which", C.c_int32),
+        ("seam_after", C.c_int32), ("which", C.c_int32), ("sink_tokens", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -221,8 +221,8 @@ def kvb_assemble(ctx, table: RequestTable, stream=None, check: bool = True) -> i
 
 
 def kvb_deviation_topk(ctx, table: RequestTable, ratio: float, k_override: int, seam_before: int, seam_after: int,
-                       which: int, out: SelectionTable, stream=None, check: bool = True) -> int:
-    p = kvb_select_params(ratio, k_override, seam_before, seam_after, which)
+                       which: int, out: SelectionTable, stream=None, check: bool = True, sink_tokens: int = 0) -> int:
+    p = kvb_select_params(ratio, k_override, seam_before, seam_after, which, sink_tokens, 0)
     st = lib().kvb_deviation_topk(ctx, table.array, table.n, C.byref(p), out.array, _stream(stream))
     return _check(ctx, st) if check else st
 

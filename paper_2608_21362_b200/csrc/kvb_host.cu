@@ -312,7 +312,7 @@ int kvb_deviation_topk(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
   if (st0 != KVB_OK) return st0;
   if (n_req == 0) return KVB_OK;
   if (!p || !out) return fail(c, KVB_ERR_INVALID_ARG, "NULL select params or outputs");
-  if ((p->which & 3) == 0 || (p->which & ~3) || p->seam_before < 0 || p->seam_after < 0 ||
+  if ((p->which & 3) == 0 || (p->which & ~3) || p->seam_before < 0 || p->seam_after < 0 || p->sink_tokens < 0 ||
       (p->k_override < 0 && !(p->ratio >= 0.0 && p->ratio <= 1.0)))
     return fail(c, KVB_ERR_INVALID_ARG, "bad select params");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -356,6 +356,12 @@ int kvb_deviation_topk(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
       SeamWindow w;
       w.lo = pos - p->seam_before < 0 ? 0 : pos - p->seam_before;
       w.hi = pos + p->seam_after > q.T ? q.T : pos + p->seam_after;
+      sw[n_seams++] = w;
+    }
+    if (p->sink_tokens > 0) {  // attention sinks: the first s positions, one more window
+      SeamWindow w;
+      w.lo = 0;
+      w.hi = p->sink_tokens > q.T ? q.T : p->sink_tokens;
       sw[n_seams++] = w;
     }
     d.n_seams = n_seams - d.seam_offset;

@@ -101,6 +101,27 @@ def test_selection_at_its_size_limits():
         B.kvb_destroy(ctx)
 
 
+def test_attention_sink_tokens_join_the_selection():
+    wl = synth.workload(0)
+    sh = wl.shape
+    reqs = prepare(wl)
+    (r,) = reqs
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        k = B.kvb_select_count(r.plan.T, 0.15)
+        sel = B.SelectionTable([r.plan.T], [k], [r.plan.T], DEV)
+        B.kvb_deviation_topk(ctx, tbl, 0.15, -1, 16, 0, 3, sel, sink_tokens=4)
+        B.kvb_last_status(ctx)
+        rank = sel.rank[0].cpu().numpy()[:k]
+        want = oracle.seam_select(rank, [c.plan.new_pos for c in r.chunks], [c.plan.mode for c in r.chunks], r.plan.T, 16, 0, sinks=4)
+        n = int(sel.n_sel[0])
+        assert np.array_equal(sel.sel[0].cpu().numpy()[:n], want) and {0, 1, 2, 3} <= set(want.tolist())
+        assert B.kvb_deviation_topk(ctx, tbl, 0.15, -1, 16, 0, 3, sel, check=False, sink_tokens=-1) == B.KVB_ERR_INVALID_ARG
+    finally:
+        B.kvb_destroy(ctx)
+
+
 def test_empty_selection_and_wide_overlapping_seam_windows():
     wl = synth.workload(0)
     sh = wl.shape

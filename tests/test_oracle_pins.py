@@ -342,6 +342,17 @@ def test_seam_windows_closed_form():
     assert list(sel) == sorted(set(want) | {300, 120, 5}) and len(sel) == 6 * 16 + 2
 
 
+def test_sink_tokens_are_always_selected():
+    T, C = 512, 128
+    pos, mode = np.arange(0, T, C), np.array([0, 0, 2, 2])  # seams at 256 and 384 only
+    none = np.zeros(0, np.int32)
+    assert list(oracle.seam_select(none, pos, mode, T, 0, 0, sinks=4)) == [0, 1, 2, 3]
+    sel = oracle.seam_select(np.array([2, 300], np.int32), pos, mode, T, 16, 0, sinks=4)
+    assert list(sel) == sorted({0, 1, 2, 3, 300} | set(range(240, 256)) | set(range(368, 384)))
+    assert list(oracle.seam_select(none, pos, mode, T, 0, 0, sinks=10**6)) == list(range(T))  # clamped at T
+    assert list(oracle.seam_select(none, pos, mode, T, 0, 0)) == []
+
+
 # ------------------------------------------------------------------ Eq. 2
 def _attn_case(L=2, T=24, Hq=4, Hkv=2, d=16, dtype=1, seed=9):
     r = np.random.default_rng(seed)
