@@ -147,13 +147,21 @@ class Replica:
         return n
 
 
+ONE_PASS = True  # stitch and deviation sums in one kernel (kvb_assemble_select); --path two-call uses the separate calls
+
+
 def step(B, ctx, rep, sp, scale, events=None):
     if events:
         events[0].record()
-    B.kvb_assemble(ctx, rep.tbl)
-    if events:
-        events[1].record()
-    B.kvb_deviation_topk(ctx, rep.tbl, sp.ratio, sp.k_override, sp.seam_before, sp.seam_after, sp.which, rep.sel)
+    if ONE_PASS:
+        B.kvb_assemble_select(ctx, rep.tbl, sp.ratio, sp.k_override, sp.seam_before, sp.seam_after, sp.which, rep.sel)
+        if events:
+            events[1].record()
+    else:
+        B.kvb_assemble(ctx, rep.tbl)
+        if events:
+            events[1].record()
+        B.kvb_deviation_topk(ctx, rep.tbl, sp.ratio, sp.k_override, sp.seam_before, sp.seam_after, sp.which, rep.sel)
     if events:
         events[2].record()
     B.kvb_selective_attn(ctx, rep.tbl, rep.sel, rep.q, rep.out, scale)
@@ -258,10 +266,13 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOADS))
     ap.add_argument("--replicas", type=int, default=0, help="independent copies rotated through (0 = auto)")
     ap.add_argument("--batch", type=int, default=1, help="requests per step: the workload's request list repeated this many times")
+    ap.add_argument("--path", default="one-pass", choices=["one-pass", "two-call"], help="kvb_assemble_select, or kvb_assemble + kvb_deviation_topk")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    global ONE_PASS
+    ONE_PASS = args.path == "one-pass"
     wl = synth.workload(WORKLOADS[args.workload])
     if args.batch > 1:
         wl = synth.Workload("%s_x%d" % (wl.name, args.batch), wl.seed, wl.shape, wl.requests * args.batch, wl.select, wl.sigma_bulk, wl.sigma_seam, wl.seam_tokens)
@@ -411,11 +422,21 @@ def main():
     value = job_throughput(world, n_tok, ms_step)
     long_run = ms_total > 1000.0
     tensor_peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
-    stages = {
-        "assemble": {"bound": "hbm", "ms": stage_ms[0], "achieved": asm_bytes / stage_ms[0] / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s", "algorithmic_bytes": asm_bytes},
-        "deviation_topk": {"bound": "hbm", "ms": stage_ms[1], "achieved": dev_bytes / stage_ms[1] / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s", "algorithmic_bytes": dev_bytes},
-        "selective_attn": {"bound": "tensor", "ms": stage_ms[2], "achieved": attn_flops / stage_ms[2] / 1e9, "peak": tensor_peak, "unit": "TFLOP/s", "algorithmic_flops": attn_flops},
-    }
+    attn_stage = {"bound": "tensor", "ms": stage_ms[2], "achieved": attn_flops / stage_ms[2] / 1e9, "peak": tensor_peak, "unit": "TFLOP/s", "algorithmic_flops": attn_flops}
+    if ONE_PASS:  # stitch + deviation sums + selection behind one call
+        one_bytes = sum(synth.one_pass_bytes(sh, r.plan, sp.which) for r in reps[0].reqs)
+        ms01 = stage_ms[0] + stage_ms[1]
+        stages = {
+            "assemble_select": {"bound": "hbm", "ms": ms01, "achieved": one_bytes / ms01 / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s", "algorithmic_bytes": one_bytes,
+                                "two_call_bytes": asm_bytes + dev_bytes},
+            "selective_attn": attn_stage,
+        }
+    else:
+        stages = {
+            "assemble": {"bound": "hbm", "ms": stage_ms[0], "achieved": asm_bytes / stage_ms[0] / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s", "algorithmic_bytes": asm_bytes},
+            "deviation_topk": {"bound": "hbm", "ms": stage_ms[1], "achieved": dev_bytes / stage_ms[1] / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s", "algorithmic_bytes": dev_bytes},
+            "selective_attn": attn_stage,
+        }
     for s in stages.values():
         s["frac"] = s["achieved"] / s["peak"]
     top = max(stages, key=lambda k: stages[k]["ms"])
@@ -435,7 +456,8 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if sh.kv_dtype == "bf16" else "fp16", "data": "synthetic",
         "config": {
-            "workload": wl.name, "requests_per_step": len(wl.requests), "tokens_per_step": n_tok, "layers": sh.L, "q_heads": sh.Hq,
+            "workload": wl.name, "path": "kvb_assemble_select + kvb_selective_attn" if ONE_PASS else "kvb_assemble + kvb_deviation_topk + kvb_selective_attn",
+            "requests_per_step": len(wl.requests), "tokens_per_step": n_tok, "layers": sh.L, "q_heads": sh.Hq,
             "kv_heads": sh.Hkv, "head_dim": sh.d, "chunk_tokens": sh.C, "select_ratio": sp.ratio, "seam_window": [sp.seam_before, sp.seam_after],
             "parallelism": "replicas only (one independent stream of requests per GPU)" if world > 1 else "single GPU",
             "l2": "inputs larger than L2: %d replicas rotated, %.0f MB resident" % (n_rep, footprint / 1e6),

@@ -158,6 +158,17 @@ int kvb_assemble(kvb_ctx* ctx, const kvb_request* reqs, int n_req, void* cuda_st
 int kvb_deviation_topk(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_select_params* params,
                        const kvb_selection* out, void* cuda_stream);
 
+/* kvb_assemble followed by kvb_deviation_topk, with the deviation sums taken
+ * while the stitched rows are still in registers, so kv_buf is written once and
+ * never read back and `fresh` is read once (Prompt Assembly + Algorithm 2 steps
+ * 2-3 + the token set of Algorithm 1 in one pass over the chunk store).
+ * Writes the same kv_buf as kvb_assemble; delta agrees with the two-call
+ * path to float32 rounding of the per-row sums (a few 1e-7), and rank / sel
+ * are the selection of this call's delta.  Arguments and errors as for the
+ * two calls; chunks need their payload pointers. */
+int kvb_assemble_select(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_select_params* params,
+                        const kvb_selection* out, void* cuda_stream);
+
 /* Causal attention (Eq. 2) of the selected rows only.  q[r], out[r]: device,
  * [L][sel_capacity][Hq][d] in kv_dtype; row i belongs to position sel[i] and
  * attends keys 0..sel[i] of kv_buf; query head hq reads KV head hq/(Hq/Hkv).

@@ -97,6 +97,7 @@ def lib():
         L.kvb_destroy.argtypes = [vp]
         L.kvb_assemble.argtypes = [vp, C.POINTER(kvb_request), C.c_int, vp]
         L.kvb_deviation_topk.argtypes = [vp, C.POINTER(kvb_request), C.c_int, C.POINTER(kvb_select_params), C.POINTER(kvb_selection), vp]
+        L.kvb_assemble_select.argtypes = L.kvb_deviation_topk.argtypes
         L.kvb_selective_attn.argtypes = [vp, C.POINTER(kvb_request), C.c_int, C.POINTER(kvb_selection), C.POINTER(vp), C.POINTER(vp), C.c_float, vp]
         L.kvb_quantize_chunk.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp]
         L.kvb_select_count.argtypes = [C.c_int, C.c_double]
@@ -224,6 +225,13 @@ def kvb_deviation_topk(ctx, table: RequestTable, ratio: float, k_override: int, 
                        which: int, out: SelectionTable, stream=None, check: bool = True, sink_tokens: int = 0) -> int:
     p = kvb_select_params(ratio, k_override, seam_before, seam_after, which, sink_tokens, 0)
     st = lib().kvb_deviation_topk(ctx, table.array, table.n, C.byref(p), out.array, _stream(stream))
+    return _check(ctx, st) if check else st
+
+
+def kvb_assemble_select(ctx, table: RequestTable, ratio: float, k_override: int, seam_before: int, seam_after: int,
+                        which: int, out: SelectionTable, stream=None, check: bool = True, sink_tokens: int = 0) -> int:
+    p = kvb_select_params(ratio, k_override, seam_before, seam_after, which, sink_tokens, 0)
+    st = lib().kvb_assemble_select(ctx, table.array, table.n, C.byref(p), out.array, _stream(stream))
     return _check(ctx, st) if check else st
 
 

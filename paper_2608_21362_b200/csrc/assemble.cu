@@ -14,6 +14,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "deviation_math.cuh"
 #include "f32x2.cuh"
 #include "kvb_internal.h"
 
@@ -76,6 +77,7 @@ template <typename T>
 struct Pack;
 template <>
 struct Pack<__nv_bfloat16> {
+  static constexpr int DT = KVB_DT_BF16;
   static __device__ __forceinline__ uint32_t two(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -86,6 +88,7 @@ struct Pack<__nv_bfloat16> {
 };
 template <>
 struct Pack<__half> {
+  static constexpr int DT = KVB_DT_F16;
   static __device__ __forceinline__ uint32_t two(float a, float b) {
     __half2 v = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -96,12 +99,15 @@ struct Pack<__half> {
   }
 };
 
+// rounds four values to the output type, stores them and returns the stored words
 template <typename OutT>
-__device__ __forceinline__ void store4(OutT* p, const uint64_t (&v)[2]) {
+__device__ __forceinline__ uint2 store4(OutT* p, const uint64_t (&v)[2]) {
   float a, b, c, e;
   f2_unpack(v[0], a, b);
   f2_unpack(v[1], c, e);
-  *reinterpret_cast<uint2*>(p) = make_uint2(Pack<OutT>::two(a, b), Pack<OutT>::two(c, e));
+  const uint2 w = make_uint2(Pack<OutT>::two(a, b), Pack<OutT>::two(c, e));
+  *reinterpret_cast<uint2*>(p) = w;
+  return w;
 }
 
 __device__ __forceinline__ void copy_rows(uint8_t* dst, const uint8_t* src, size_t bytes, int tid) {
@@ -120,10 +126,37 @@ __device__ __forceinline__ void copy_rows(uint8_t* dst, const uint8_t* src, size
   for (; i < n; i += kThreads) d[i] = __ldcs(s + i);
 }
 
-template <typename OutT>
+// Copy of `rows` 256-byte (token, head) rows (a multiple of 32) that also accumulates each row's
+// deviation term against the fresh tensor: a half-warp per row, two rows per pass.
+// acc_tok points at the accumulator of the first row's token.
+template <int DT>
+__device__ __forceinline__ void copy_rows_dev(uint8_t* dst, const uint8_t* src, const uint8_t* fresh, int rows, int H,
+                                              int tid, unsigned long long* acc_tok) {
+  const int lane = tid & 31, s = lane >> 4, ln = lane & 15;
+  const int hw = (tid >> 5) * 2 + s;
+  const bool heads_paired = (H & 1) == 0;  // rows 2w, 2w+1 of a warp belong to one token
+  for (int ua = hw; ua < rows; ua += 32) {
+    const int ub = ua + 16;
+    const size_t oa = (size_t)ua * 256 + (size_t)ln * 16, ob = (size_t)ub * 256 + (size_t)ln * 16;
+    const uint4 a0 = __ldcs(reinterpret_cast<const uint4*>(src + oa)), a1 = __ldcs(reinterpret_cast<const uint4*>(src + ob));
+    const uint4 b0 = __ldcs(reinterpret_cast<const uint4*>(fresh + oa)), b1 = __ldcs(reinterpret_cast<const uint4*>(fresh + ob));
+    *reinterpret_cast<uint4*>(dst + oa) = a0;
+    *reinterpret_cast<uint4*>(dst + ob) = a1;
+    float sa[3], sb[3];
+    row_sums<DT>(a0, b0, sa[0], sa[1], sa[2]);
+    row_sums<DT>(a1, b1, sb[0], sb[1], sb[2]);
+    long long fx = pair_terms_fixed(sa, sb, ln, true, true);
+    if (heads_paired) fx += __shfl_xor_sync(0xffffffffu, fx, 16);
+    if ((ln & 7) == 0 && (!heads_paired || s == 0)) atomicAdd(acc_tok + ((ln & 8) ? ub : ua) / H, (unsigned long long)fx);
+  }
+}
+
+// DEV = true adds the deviation of every written row against the fresh tensor (Algorithm 2, step 2)
+// to acc[token]: K rows when which & 1, V rows when which & 2.
+template <typename OutT, bool DEV>
 __global__ void __launch_bounds__(kThreads, 3)
     assemble_kernel(const ChunkDesc* __restrict__ chunks, const float2* __restrict__ cs_table, ModelDims m,
-                    uint32_t* __restrict__ status) {
+                    uint32_t* __restrict__ status, int which, unsigned long long* __restrict__ acc) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) uint64_t bars[kParts + 1];
 
@@ -146,14 +179,20 @@ __global__ void __launch_bounds__(kThreads, 3)
   const size_t out_bytes = (size_t)C * row_elems * 2;
   const size_t layer_out_bytes = (size_t)m.C * row_elems * 2;
 
-  // ---- rows that are plain copies: FRESH chunks; unquantised values; unquantised keys that do not move
+  const bool dev_on = DEV && (which & (kv ? 2 : 1));
+  unsigned long long* acc_tok = DEV ? acc + cd.tok_offset + cd.new_pos + tb : nullptr;  // this CTA's first token
+
+  // ---- rows that are plain copies: FRESH chunks (deviation 0); unquantised values; unquantised keys that do not move
   if (cd.mode == KVB_MODE_FRESH) {
     copy_rows(reinterpret_cast<uint8_t*>(dst), cd.fresh + dst_off * 2, out_bytes, tid);
     return;
   }
   if (cd.mode == KVB_MODE_FP16 && (kv == 1 || cd.delta_pos == 0)) {
-    copy_rows(reinterpret_cast<uint8_t*>(dst), (kv ? cd.v_src : cd.k_src) + (size_t)l * layer_out_bytes + (size_t)tb * row_elems * 2,
-              out_bytes, tid);
+    const uint8_t* src = (kv ? cd.v_src : cd.k_src) + (size_t)l * layer_out_bytes + (size_t)tb * row_elems * 2;
+    if (dev_on)
+      copy_rows_dev<Pack<OutT>::DT>(reinterpret_cast<uint8_t*>(dst), src, cd.fresh + dst_off * 2, C * H, H, tid, acc_tok);
+    else
+      copy_rows(reinterpret_cast<uint8_t*>(dst), src, out_bytes, tid);
     return;
   }
 
@@ -239,6 +278,35 @@ __global__ void __launch_bounds__(kThreads, 3)
   };
   const float bias = bits == 4 ? 16.f : 0.f;  // what the 4-bit unpacking adds to every code
 
+  // waits (bounded) for the part of the codes that token t lies in; false = give up
+  auto part_ready = [&](int t) {
+    const int part = t / tok_per_part;
+    if (part != ready_part) {
+      ok = ok && mbar_wait(&bars[1 + part], 0);
+      ready_part = part;
+    }
+    if (DEV) ok = __all_sync(0xffffffffu, ok);  // the deviation's shuffles need the whole warp
+    return ok;
+  };
+  // Deviation terms of tokens t and t+1 of this half-warp's head: the stored words are still in
+  // registers, the fresh row's matching 2 x 8 bytes per lane come from global memory.
+  const uint8_t* fresh_rows = cd.fresh + dst_off * 2;
+  auto dev_pair = [&](int t, const uint2& wl0, const uint2& wh0, const uint2& wl1, const uint2& wh1) {
+    const uint8_t* f0 = fresh_rows + (size_t)(t * H + h) * (d * 2) + 8 * ln;
+    const uint8_t* f1 = f0 + (size_t)H * (d * 2);
+    const uint2 fl0 = __ldcs(reinterpret_cast<const uint2*>(f0)), fh0 = __ldcs(reinterpret_cast<const uint2*>(f0 + 128));
+    const uint2 fl1 = __ldcs(reinterpret_cast<const uint2*>(f1)), fh1 = __ldcs(reinterpret_cast<const uint2*>(f1 + 128));
+    const uint32_t a0[4] = {wl0.x, wl0.y, wh0.x, wh0.y}, b0[4] = {fl0.x, fl0.y, fh0.x, fh0.y};
+    const uint32_t a1[4] = {wl1.x, wl1.y, wh1.x, wh1.y}, b1[4] = {fl1.x, fl1.y, fh1.x, fh1.y};
+    float sa[3], sb[3];
+    row_sums4<Pack<OutT>::DT>(a0, b0, sa[0], sa[1], sa[2]);
+    row_sums4<Pack<OutT>::DT>(a1, b1, sb[0], sb[1], sb[2]);
+    long long fx = pair_terms_fixed(sa, sb, ln, true, true);
+    const bool heads_paired = (H & 1) == 0;  // the warp's two half-warps hold two heads of the same tokens
+    if (heads_paired) fx += __shfl_xor_sync(0xffffffffu, fx, 16);
+    if ((ln & 7) == 0 && (!heads_paired || s == 0)) atomicAdd(acc_tok + t + (ln >> 3), (unsigned long long)fx);
+  };
+
   if (!kv) {
     // ------------------------------ keys
     uint64_t A_lo[2], B_lo[2], C_lo[2], A_hi[2], B_hi[2], C_hi[2];
@@ -253,15 +321,7 @@ __global__ void __launch_bounds__(kThreads, 3)
     const uint64_t s2[2] = {f2_pack(cs_s[0], cs_s[1]), f2_pack(cs_s[2], cs_s[3])};
     const uint64_t ns2[2] = {f2_pack(-cs_s[0], -cs_s[1]), f2_pack(-cs_s[2], -cs_s[3])};
     int cur_group = -1;
-#pragma unroll 2
-    for (int tt = 0; tt < tok_per; ++tt) {
-      const int t = t0 + tt;
-      const int part = t / tok_per_part;
-      if (part != ready_part) {
-        ok = ok && mbar_wait(&bars[1 + part], 0);
-        ready_part = part;
-      }
-      if (!ok) break;
+    auto key_row = [&](int t, uint2& wl, uint2& wh) {
       const int u = t * H + h;
       OutT* orow = dst + (size_t)u * d;
       uint64_t ol[2], oh[2];
@@ -311,20 +371,20 @@ __global__ void __launch_bounds__(kThreads, 3)
           oh[i] = f2_fma(A_hi[i], qh[i], f2_fma(B_hi[i], ql[i], C_hi[i]));
         }
       }
-      store4(orow + 4 * ln, ol);
-      store4(orow + 64 + 4 * ln, oh);
+      wl = store4(orow + 4 * ln, ol);
+      wh = store4(orow + 64 + 4 * ln, oh);
+    };
+    for (int tt = 0; tt < tok_per; tt += 2) {  // tok_per is even and a pair never straddles a part
+      const int t = t0 + tt;
+      if (!part_ready(t)) break;
+      uint2 wl0, wh0, wl1, wh1;
+      key_row(t, wl0, wh0);
+      key_row(t + 1, wl1, wh1);
+      if (dev_on) dev_pair(t, wl0, wh0, wl1, wh1);
     }
   } else {
     // ------------------------------ values (INT8 / INT4 only; never rotated)
-#pragma unroll 2
-    for (int tt = 0; tt < tok_per; ++tt) {
-      const int t = t0 + tt;
-      const int part = t / tok_per_part;
-      if (part != ready_part) {
-        ok = ok && mbar_wait(&bars[1 + part], 0);
-        ready_part = part;
-      }
-      if (!ok) break;
+    auto value_row = [&](int t, uint2& wl, uint2& wh) {
       const int u = t * H + h;
       OutT* orow = dst + (size_t)u * d;
       float s_lo, m_lo, s_hi, m_hi;
@@ -345,8 +405,16 @@ __global__ void __launch_bounds__(kThreads, 3)
         ol[i] = f2_fma(ql[i], sl2, ml2);
         oh[i] = f2_fma(qh[i], sh2, mh2);
       }
-      store4(orow + 4 * ln, ol);
-      store4(orow + 64 + 4 * ln, oh);
+      wl = store4(orow + 4 * ln, ol);
+      wh = store4(orow + 64 + 4 * ln, oh);
+    };
+    for (int tt = 0; tt < tok_per; tt += 2) {
+      const int t = t0 + tt;
+      if (!part_ready(t)) break;
+      uint2 wl0, wh0, wl1, wh1;
+      value_row(t, wl0, wh0);
+      value_row(t + 1, wl1, wh1);
+      if (dev_on) dev_pair(t, wl0, wh0, wl1, wh1);
     }
   }
 
@@ -390,10 +458,13 @@ size_t assemble_smem_bytes(const ModelDims& m, int mode) {
 }
 
 cudaError_t assemble_configure(size_t max_smem) {
-  cudaError_t e = cudaFuncSetAttribute(assemble_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)max_smem);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(assemble_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+  const void* fns[4] = {(const void*)assemble_kernel<__nv_bfloat16, false>, (const void*)assemble_kernel<__nv_bfloat16, true>,
+                        (const void*)assemble_kernel<__half, false>, (const void*)assemble_kernel<__half, true>};
+  for (const void* f : fns) {
+    cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const double* inv_freq, int half_d,
@@ -404,12 +475,20 @@ cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const doubl
 }
 
 cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
-                            size_t smem_bytes, uint32_t* status, cudaStream_t st) {
+                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, cudaStream_t st) {
   const unsigned grid = (unsigned)n_chunks * m.L * 2 * assemble_split(m.Hkv);
-  if (m.dtype == KVB_DT_BF16)
-    assemble_kernel<__nv_bfloat16><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status);
-  else
-    assemble_kernel<__half><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status);
+  const bool dev = acc != nullptr && (which & 3);
+  if (m.dtype == KVB_DT_BF16) {
+    if (dev)
+      assemble_kernel<__nv_bfloat16, true><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, which, acc);
+    else
+      assemble_kernel<__nv_bfloat16, false><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, 0, nullptr);
+  } else {
+    if (dev)
+      assemble_kernel<__half, true><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, which, acc);
+    else
+      assemble_kernel<__half, false><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, 0, nullptr);
+  }
   return cudaGetLastError();
 }
 

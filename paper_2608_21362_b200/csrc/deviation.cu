@@ -12,6 +12,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "deviation_math.cuh"
 #include "f32x2.cuh"
 #include "kvb_internal.h"
 
@@ -20,42 +21,6 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kTileTokens = 64;
-constexpr float kFixScale = 1099511627776.0f;  // 2^40
-
-// One 32-bit word holds two 16-bit values: unpack them into a packed float32 pair.
-template <int DT>
-__device__ __forceinline__ uint64_t unpack_pair(uint32_t w) {
-  if (DT == KVB_DT_BF16) return f2_pack(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
-  const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&w));
-  return f2_pack(t.x, t.y);
-}
-
-// ||a-b||^2, ||a||^2, ||b||^2 over this lane's 8 elements, in packed float32 pairs
-template <int DT>
-__device__ __forceinline__ void row_sums(const uint4& a, const uint4& b, float& d2, float& na2, float& nb2) {
-  const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
-  uint64_t sd = 0ull, sa = 0ull, sb = 0ull;  // bit pattern of (+0, +0)
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const uint64_t x = unpack_pair<DT>(aw[i]), y = unpack_pair<DT>(bw[i]);
-    const uint64_t df = f2_sub(x, y);
-    sd = f2_fma(df, df, sd);
-    sa = f2_fma(x, x, sa);
-    sb = f2_fma(y, y, sb);
-  }
-  d2 = f2_hsum(sd);
-  na2 = f2_hsum(sa);
-  nb2 = f2_hsum(sb);
-}
-
-__device__ __forceinline__ float one_minus_cos(float d2, float na2, float nb2) {
-  if (d2 == 0.f) return 0.f;                 // identical rows (zero rows included): cos = 1
-  if (na2 == 0.f || nb2 == 0.f) return 1.f;  // one zero row: cos = 0
-  const float na = sqrtf(na2), nb = sqrtf(nb2);
-  const float dn = (na2 - nb2) / (na + nb);
-  const float r = (d2 - dn * dn) / (2.f * na * nb);
-  return fminf(fmaxf(r, 0.f), 2.f);
-}
 
 // grid (tiles over all requests, L).  A tile is kTileTokens consecutive positions of one request.
 template <int DT>

@@ -221,7 +221,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
 
   const size_t a1 = sizeof(ChunkDesc) * (size_t)limits->max_chunks_total;
   const size_t a2 = (sizeof(ReqDesc) + 256) * (size_t)limits->max_requests + 128 + sizeof(SeamWindow) * (size_t)limits->max_chunks_total;
-  c->arena_bytes = ((a1 > a2 ? a1 : a2) + 255) & ~(size_t)255;
+  c->arena_bytes = ((a1 + 255) & ~(size_t)255) + ((a2 + 255) & ~(size_t)255);  // the fused call uploads both tables
   KVB_CUDA(c, cudaMalloc(&c->arena_dev, c->arena_bytes));
   KVB_CUDA(c, cudaMallocHost(&c->staging, c->arena_bytes * kSlots));
   for (int s = 0; s < kSlots; ++s) KVB_CUDA(c, cudaEventCreateWithFlags(&c->slot_done[s], cudaEventDisableTiming));
@@ -259,22 +259,14 @@ int kvb_last_status(kvb_ctx* c) {
   return KVB_OK;
 }
 
-int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stream) {
-  int n_chunks = 0;
-  int64_t n_tok = 0;
-  const int st0 = check_batch(c, reqs, n_req, true, &n_chunks, &n_tok);
-  if (st0 != KVB_OK) return st0;
-  if (n_req == 0) return KVB_OK;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  KVB_CUDA(c, cudaSetDevice(c->device));
+}  // extern "C"
 
-  uint8_t* host = nullptr;
-  const int slot_code = take_slot(c, &host);
-  if (slot_code >= 0) return slot_code;
-  const int slot = -slot_code - 1;
-  ChunkDesc* cd = reinterpret_cast<ChunkDesc*>(host);
+namespace {
+
+// One ChunkDesc per chunk of the batch, in request order; returns the largest shared-memory need.
+size_t pack_chunks(kvb_ctx* c, const kvb_request* reqs, int n_req, ChunkDesc* cd) {
   size_t smem = 0;
-  int n = 0;
+  int n = 0, tok = 0;
   for (int r = 0; r < n_req; ++r) {
     for (int i = 0; i < reqs[r].n_chunks; ++i, ++n) {
       const kvb_chunk& k = reqs[r].chunks[i];
@@ -289,41 +281,31 @@ int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stre
       d.new_pos = k.new_pos;
       d.delta_pos = k.mode == KVB_MODE_FRESH ? 0 : k.new_pos - k.orig_pos;
       d.mode = k.mode;
+      d.tok_offset = tok;
       cd[n] = d;
       const size_t s = assemble_smem_bytes(c->dims, k.mode);
       if (s > smem) smem = s;
     }
+    tok += reqs[r].T;
   }
-  const int up = upload(c, slot, host, sizeof(ChunkDesc) * (size_t)n, st);
-  if (up != KVB_OK) return up;
-  c->last_stream = st;
-  const ChunkDesc* cd_dev = reinterpret_cast<const ChunkDesc*>(c->arena_dev);
-  KVB_CUDA(c, launch_rope_table(cd_dev, n, c->inv_freq, c->model.d / 2, c->cs_table, st));
-  KVB_CUDA(c, launch_assemble(cd_dev, n, c->cs_table, c->dims, smem, c->status_dev, st));
-  c->launches += 2;
-  return KVB_OK;
+  return smem;
 }
 
-int kvb_deviation_topk(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_select_params* p,
-                       const kvb_selection* out, void* cuda_stream) {
-  int n_chunks = 0;
-  int64_t n_tok = 0;
-  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
-  if (st0 != KVB_OK) return st0;
-  if (n_req == 0) return KVB_OK;
+int check_select_args(kvb_ctx* c, const kvb_select_params* p, const kvb_selection* out) {
   if (!p || !out) return fail(c, KVB_ERR_INVALID_ARG, "NULL select params or outputs");
   if ((p->which & 3) == 0 || (p->which & ~3) || p->seam_before < 0 || p->seam_after < 0 || p->sink_tokens < 0 ||
       (p->k_override < 0 && !(p->ratio >= 0.0 && p->ratio <= 1.0)))
     return fail(c, KVB_ERR_INVALID_ARG, "bad select params");
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  KVB_CUDA(c, cudaSetDevice(c->device));
+  return KVB_OK;
+}
 
-  uint8_t* host = nullptr;
-  const int slot_code = take_slot(c, &host);
-  if (slot_code >= 0) return slot_code;
-  const int slot = -slot_code - 1;
-  ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
-  SeamWindow* sw = reinterpret_cast<SeamWindow*>(host + sizeof(ReqDesc) * (size_t)n_req);
+struct SelectExtent {
+  int tiles = 0, n_seams = 0, max_T = 0, max_k = 0;
+};
+
+// One ReqDesc per request plus the batch's window list (seams, then the sink window, per request).
+int pack_selection(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_select_params* p, const kvb_selection* out,
+                   ReqDesc* rd, SeamWindow* sw, SelectExtent* ext) {
   const int tile_tok = deviation_tile_tokens();
   int tiles = 0, tok = 0, n_seams = 0, max_T = 0, max_k = 0;
   for (int r = 0; r < n_req; ++r) {
@@ -371,21 +353,124 @@ int kvb_deviation_topk(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
     if (q.T > max_T) max_T = q.T;
     if (k > max_k) max_k = k;
   }
+  ext->tiles = tiles, ext->n_seams = n_seams, ext->max_T = max_T, ext->max_k = max_k;
+  return KVB_OK;
+}
+
+int clear_acc_if_dirty(kvb_ctx* c, cudaStream_t st) {
   if (c->acc_dirty) {
     KVB_CUDA(c, cudaMemsetAsync(c->acc, 0, (size_t)c->limits.max_tokens_total * sizeof(unsigned long long), st));
     c->acc_dirty = false;
   }
-  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req + sizeof(SeamWindow) * (size_t)n_seams, st);
+  return KVB_OK;
+}
+
+int n_deviation_terms(const kvb_ctx* c, int which) { return c->model.L * c->model.Hkv * ((which & 1) + ((which >> 1) & 1)); }
+
+}  // namespace
+
+extern "C" {
+
+int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, true, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  const size_t smem = pack_chunks(c, reqs, n_req, reinterpret_cast<ChunkDesc*>(host));
+  const int up = upload(c, slot, host, sizeof(ChunkDesc) * (size_t)n_chunks, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  const ChunkDesc* cd_dev = reinterpret_cast<const ChunkDesc*>(c->arena_dev);
+  KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, 0, nullptr, st));
+  c->launches += 2;
+  return KVB_OK;
+}
+
+int kvb_deviation_topk(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_select_params* p,
+                       const kvb_selection* out, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  const int st1 = check_select_args(c, p, out);
+  if (st1 != KVB_OK) return st1;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
+  SeamWindow* sw = reinterpret_cast<SeamWindow*>(host + sizeof(ReqDesc) * (size_t)n_req);
+  SelectExtent ext;
+  const int st2 = pack_selection(c, reqs, n_req, p, out, rd, sw, &ext);
+  if (st2 != KVB_OK) return st2;
+  const int st3 = clear_acc_if_dirty(c, st);
+  if (st3 != KVB_OK) return st3;
+  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req + sizeof(SeamWindow) * (size_t)ext.n_seams, st);
   if (up != KVB_OK) return up;
   c->last_stream = st;
   const ReqDesc* rd_dev = reinterpret_cast<const ReqDesc*>(c->arena_dev);
   const SeamWindow* sw_dev = reinterpret_cast<const SeamWindow*>(c->arena_dev + sizeof(ReqDesc) * (size_t)n_req);
   c->acc_dirty = true;  // cleared again once both kernels are in the stream
-  KVB_CUDA(c, launch_deviation(rd_dev, n_req, tiles, c->dims, p->which, c->acc, st));
-  const int n_terms = c->model.L * c->model.Hkv * ((p->which & 1) + ((p->which >> 1) & 1));
-  KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_terms, max_T, max_k, c->acc, c->status_dev, st));
+  KVB_CUDA(c, launch_deviation(rd_dev, n_req, ext.tiles, c->dims, p->which, c->acc, st));
+  KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_deviation_terms(c, p->which), ext.max_T, ext.max_k, c->acc,
+                          c->status_dev, st));
   c->acc_dirty = false;
   c->launches += 2;
+  return KVB_OK;
+}
+
+int kvb_assemble_select(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_select_params* p,
+                        const kvb_selection* out, void* cuda_stream) {
+  int n_chunks = 0;
+  int64_t n_tok = 0;
+  const int st0 = check_batch(c, reqs, n_req, true, &n_chunks, &n_tok);
+  if (st0 != KVB_OK) return st0;
+  if (n_req == 0) return KVB_OK;
+  const int st1 = check_select_args(c, p, out);
+  if (st1 != KVB_OK) return st1;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  // arena: chunk descriptors, then (256-byte aligned) request descriptors and the window list
+  const size_t rd_off = (sizeof(ChunkDesc) * (size_t)n_chunks + 255) & ~(size_t)255;
+  const size_t sw_off = rd_off + sizeof(ReqDesc) * (size_t)n_req;
+  const size_t smem = pack_chunks(c, reqs, n_req, reinterpret_cast<ChunkDesc*>(host));
+  SelectExtent ext;
+  const int st2 = pack_selection(c, reqs, n_req, p, out, reinterpret_cast<ReqDesc*>(host + rd_off),
+                                 reinterpret_cast<SeamWindow*>(host + sw_off), &ext);
+  if (st2 != KVB_OK) return st2;
+  const int st3 = clear_acc_if_dirty(c, st);
+  if (st3 != KVB_OK) return st3;
+  const int up = upload(c, slot, host, sw_off + sizeof(SeamWindow) * (size_t)ext.n_seams, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  const ChunkDesc* cd_dev = reinterpret_cast<const ChunkDesc*>(c->arena_dev);
+  const ReqDesc* rd_dev = reinterpret_cast<const ReqDesc*>(c->arena_dev + rd_off);
+  const SeamWindow* sw_dev = reinterpret_cast<const SeamWindow*>(c->arena_dev + sw_off);
+  KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+  c->acc_dirty = true;  // cleared again once both kernels are in the stream
+  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, p->which, c->acc, st));
+  KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_deviation_terms(c, p->which), ext.max_T, ext.max_k, c->acc,
+                          c->status_dev, st));
+  c->acc_dirty = false;
+  c->launches += 3;
   return KVB_OK;
 }
 

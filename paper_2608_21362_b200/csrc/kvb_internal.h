@@ -27,6 +27,8 @@ struct ChunkDesc {
   int32_t new_pos;
   int32_t delta_pos;     // new_pos - orig_pos
   int32_t mode;
+  int32_t tok_offset;    // first token of the request in the call's flat token space
+  int32_t reserved;
 };
 
 // One request, as the deviation / top-k / attention kernels see it.
@@ -58,10 +60,11 @@ struct ModelDims {
 };
 
 // ---- launchers (each defined next to its kernel) ----
+// launch_assemble: acc != NULL fuses the deviation sums (which: bit 0 keys, bit 1 values) into the stitch.
 cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const double* inv_freq, int half_d,
                               float2* cs_table, cudaStream_t st);
 cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
-                            size_t smem_bytes, uint32_t* status, cudaStream_t st);
+                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, cudaStream_t st);
 size_t assemble_smem_bytes(const ModelDims& m, int mode);
 cudaError_t assemble_configure(size_t max_smem);
 

@@ -253,6 +253,15 @@ def deviation_bytes(sh: Shape, plan: RequestPlan, which: int) -> int:
     return sh.L * nw * plan.T * sh.Hkv * sh.d * 2 * 2  # stored + fresh rows, 16-bit
 
 
+def one_pass_bytes(sh: Shape, plan: RequestPlan, which: int) -> int:
+    """Bytes of the stitch with the deviation sums taken in the same pass: the stitch's own traffic
+    plus one read of the fresh rows of every cached chunk (the stored rows are never read back, a
+    FRESH chunk's rows are a copy and deviate by nothing)."""
+    nw = (which & 1) + ((which >> 1) & 1)
+    cached = sum(1 for cp in plan.chunks if cp.mode != MODE_FRESH)
+    return assemble_bytes(sh, plan) + sh.L * nw * cached * sh.C * sh.Hkv * sh.d * 2
+
+
 def attention_flops(sh: Shape, sel) -> int:
     """Causal-useful flops only: 4*d per (query head, key) pair, keys 0..t."""
     s = int(np.sum(np.asarray(sel, dtype=np.int64) + 1))
