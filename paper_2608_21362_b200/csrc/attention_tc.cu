@@ -1,8 +1,10 @@
 // Selected-row causal attention (Eq. 2) on the 5th-generation tensor cores.
 //
-// One CTA per (layer, KV head, tile of selected tokens); a tile packs TOK = 128/rep selected
-// tokens times the rep = Hq/Hkv query heads sharing the KV head into the 128 rows of one
-// tcgen05.mma (M = 128).  Keys go by sub-blocks of 64, two streams alternating:
+// Work unit: a tile = (layer, KV head, TOK = 128/rep selected tokens) x the rep = Hq/Hkv query
+// heads sharing the KV head, i.e. the 128 rows of one tcgen05.mma (M = 128).  Persistent CTAs (two
+// per SM) draw tiles from a global counter; sub-blocks are numbered through all tiles of a CTA, so
+// the next tile's lookup, loads and first Q K^T run under the current tile's last P V and epilogue.
+// Keys go by sub-blocks of 64, two streams alternating:
 //     S = Q K^T   tcgen05.mma, Q and K from shared memory (K-major, 128-byte swizzle), S in TMEM
 //     P = exp2(scale*S - m)  by 128 threads, one TMEM lane (row) each, written back over S as bf16
 //     O += P V    tcgen05.mma, P from TMEM, V from shared memory (MN-major), O in TMEM
@@ -219,19 +221,89 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 struct __align__(8) Barriers {
-  uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], o_full;
+  uint64_t tile_full[2], tile_empty[2], q_full, q_empty, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2],
+      o_full, o_empty;
 };
+
+// What the producer hands to the other roles for one tile (a two-slot ring in shared memory).
+struct TileInfo {
+  const int32_t* sel;
+  uint8_t* out;
+  int32_t n_sel, i_base, l, hk, nsb, sel_capacity;  // nsb = 0: no more tiles
+};
+
+// What the producer knows about the tile it will load next.
+struct NextTile {
+  TileInfo ti;
+  const CUtensorMap *map_q, *map_kv;
+};
+
+// Next tile that has rows, in the order: request, then groups of rq.lhk_group (layer, KV head) pairs
+// whose K/V planes fit L2 together, inside a group tile-major from the longest tile down with the
+// group's pairs interleaved.  `drawn` is the linear tile number already drawn for this call; the
+// one after it is drawn here (persistent CTAs) so that its latency is hidden.  ti.nsb = 0: none left.
+template <bool PERSISTENT>
+__device__ __forceinline__ NextTile decode_next_tile(unsigned int& drawn, unsigned int* tile_counter, const ReqDesc* __restrict__ reqs,
+                                                     const CUtensorMap* maps, int n_req, int total_tiles, int per_tile, int TOK, int Hkv) {
+  const unsigned int kNoTile = 0xFFFFFFFFu;
+    NextTile nx;
+    nx.ti.nsb = 0;
+    nx.map_q = nx.map_kv = nullptr;
+    for (;;) {  // next tile that has rows
+      const long long lin_ll = drawn;
+      if (lin_ll >= (long long)total_tiles * per_tile) break;
+      const int lin = (int)lin_ll;
+      drawn = PERSISTENT ? atomicAdd(tile_counter, 1u) : kNoTile;
+      int lo = 0, hi = n_req - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (reqs[mid].tile_offset * per_tile <= lin) lo = mid; else hi = mid - 1;
+      }
+      const ReqDesc& rq = reqs[lo];
+      const int cap = rq.sel_capacity;
+      const int tiles_r = (cap + TOK - 1) / TOK;
+      const int idx = lin - rq.tile_offset * per_tile;
+      const int G = rq.lhk_group;
+      const int grp = idx / (G * tiles_r);
+      const int rem = idx - grp * G * tiles_r;
+      const int g_eff = min(G, per_tile - grp * G);
+      const int lhk = grp * G + rem % g_eff;
+      const int tile = tiles_r - 1 - rem / g_eff;
+      const int n_sel = min(*rq.n_sel, cap);
+      const int i_base = tile * TOK;
+      if (i_base >= n_sel) continue;
+      const int t_max = min(rq.sel[min(i_base + TOK, n_sel) - 1], rq.T - 1);
+      nx.ti.sel = rq.sel;
+      nx.ti.out = rq.out;
+      nx.ti.n_sel = n_sel;
+      nx.ti.i_base = i_base;
+      nx.ti.l = lhk / Hkv;
+      nx.ti.hk = lhk % Hkv;
+      nx.ti.nsb = max(t_max, 0) / kSubKeys + 1;  // 64-key sub-blocks to visit
+      nx.ti.sel_capacity = cap;
+      nx.map_q = maps + 2 * lo;
+      nx.map_kv = maps + 2 * lo + 1;
+      break;
+    }
+    return nx;
+}
 
 // Keys are consumed in sub-blocks of 64, alternating between two streams x = sb & 1.  Each stream has
 // its own K and V buffers (16 KB each), its own S/P columns in TMEM and its own barriers, so while the
 // softmax threads work on one stream's scores the tensor core runs the other stream's P V and the
 // next Q K^T of the stream just consumed.  Both streams accumulate into the same O.
-template <int DT>
+//
+// PERSISTENT = true: two CTAs per SM draw tiles from a global counter until they run out, and the next
+// tile's lookup, loads and first Q K^T overlap the current tile's tail (pays for short tiles, i.e.
+// short prompts).  PERSISTENT = false: one tile per CTA, the hardware scheduler hands out the tiles
+// (a little faster when tiles are long).
+template <int DT, bool PERSISTENT>
 __global__ void __launch_bounds__(kThreads, 2)
     attn_tc_kernel(const ReqDesc* __restrict__ reqs, const CUtensorMap* __restrict__ maps, int n_req, int total_tiles,
-                   ModelDims m, float scale_log2, uint32_t* __restrict__ status) {
+                   ModelDims m, float scale_log2, uint32_t* __restrict__ status, unsigned int* __restrict__ tile_counter) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ Barriers bars;
+  __shared__ TileInfo s_tiles[2];
   __shared__ uint32_t s_tmem_base;
   __shared__ uint32_t s_abort;
 
@@ -239,36 +311,6 @@ __global__ void __launch_bounds__(kThreads, 2)
   const int per_tile = m.Hkv * m.L;
   const int rep = m.Hq / m.Hkv;
   const int TOK = kRows / rep;
-  // CTA order: request, then (layer, KV head), then tiles from the longest down, so that CTAs resident
-  // together stream the same K/V planes (L2 reuse) and the long tiles start first.
-  const int lin = blockIdx.x;
-  int lo = 0, hi = n_req - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (reqs[mid].tile_offset * per_tile <= lin) lo = mid; else hi = mid - 1;
-  }
-  const ReqDesc rq = reqs[lo];
-  const int tiles_r = (rq.sel_capacity + TOK - 1) / TOK;
-  // Within a request: (layer, head) pairs go in groups of rq.lhk_group whose K/V planes fit L2
-  // together; inside a group the order is tile-major from the longest tile down (longest-first
-  // packing over the whole group), the pairs of the group interleaved.
-  const int idx = lin - rq.tile_offset * per_tile;
-  const int G = rq.lhk_group;
-  const int grp = idx / (G * tiles_r);
-  const int rem = idx - grp * G * tiles_r;
-  const int g_eff = min(G, per_tile - grp * G);
-  const int lhk = grp * G + rem % g_eff;
-  const int tile = tiles_r - 1 - rem / g_eff;
-  const int hk = lhk % m.Hkv;
-  const int l = lhk / m.Hkv;
-  const CUtensorMap* map_q = maps + 2 * lo;
-  const CUtensorMap* map_kv = maps + 2 * lo + 1;
-  const int n_sel = min(*rq.n_sel, rq.sel_capacity);
-  const int i_base = tile * TOK;
-  if (i_base >= n_sel) return;  // uniform for the CTA, before anything is allocated
-  const int T = rq.T;
-  const int t_max = min(rq.sel[min(i_base + TOK, n_sel) - 1], T - 1);
-  const int nsb = t_max / kSubKeys + 1;  // 64-key sub-blocks to visit
 
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t* sQ = smem;                   // 128 rows: two 64-wide boxes of 16 KB
@@ -276,9 +318,20 @@ __global__ void __launch_bounds__(kThreads, 2)
   uint8_t* sV = smem + 2 * kTileBytes;  // same
   volatile uint32_t* abort_flag = &s_abort;
 
-  if (tid == 0) {
-    mbar_init(&bars.q_full, 1);
+  // The producer thread looks up its first tile before the CTA-wide sync, under the barrier
+  // initialisation and the TMEM allocation (done by other warps).
+  unsigned int drawn = 0xFFFFFFFFu;  // only the producer thread draws
+  if (tid == 0) drawn = PERSISTENT ? atomicAdd(tile_counter, 1u) : blockIdx.x;
+  auto decode_next = [&]() { return decode_next_tile<PERSISTENT>(drawn, tile_counter, reqs, maps, n_req, total_tiles, per_tile, TOK, m.Hkv); };
+  NextTile next;
+  next.ti.nsb = 0;
+  next.map_q = next.map_kv = nullptr;
+  if (tid == 0) next = decode_next();
+
+  if (tid == 64) {
     for (int x = 0; x < 2; ++x) {
+      mbar_init(&bars.tile_full[x], 1);
+      mbar_init(&bars.tile_empty[x], 129);  // the MMA thread and the 128 softmax threads
       mbar_init(&bars.k_full[x], 1);
       mbar_init(&bars.k_empty[x], 1);
       mbar_init(&bars.v_full[x], 1);
@@ -286,7 +339,10 @@ __global__ void __launch_bounds__(kThreads, 2)
       mbar_init(&bars.s_full[x], 1);
       mbar_init(&bars.p_full[x], 128);
     }
+    mbar_init(&bars.q_full, 1);
+    mbar_init(&bars.q_empty, 1);
     mbar_init(&bars.o_full, 1);
+    mbar_init(&bars.o_empty, 128);
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -304,38 +360,64 @@ __global__ void __launch_bounds__(kThreads, 2)
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      tensormap_acquire(map_q);
-      tensormap_acquire(map_kv);
-      mbar_expect_tx(&bars.q_full, kTileBytes);
-      tma_load_4d(sQ, map_q, 0, hk * rep, i_base, l, &bars.q_full);
-      tma_load_4d(sQ + kHalfBytes, map_q, 64, hk * rep, i_base, l, &bars.q_full);
-      // Loads are issued in the order their buffers come free: K(sb+2) as soon as S(sb) has read
-      // K(sb), V(sb) as soon as P V(sb-2) has read V(sb-2):  K0 K1 | V0 K2 | V1 K3 | ...
-      auto load_k = [&](int sb) {
-        const int x = sb & 1;
-        mbar_expect_tx(&bars.k_full[x], kSubBytes);
-        tma_load_5d(sK + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
-        tma_load_5d(sK + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
-      };
-      auto load_v = [&](int sb) {
-        const int x = sb & 1;
-        mbar_expect_tx(&bars.v_full[x], kSubBytes);
-        tma_load_5d(sV + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
-        tma_load_5d(sV + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
-      };
-      load_k(0);
-      if (nsb > 1) load_k(1);
+      // Tiles come from a global counter in the order: request, then groups of rq.lhk_group (layer,
+      // KV head) pairs whose K/V planes fit L2 together, inside a group tile-major from the longest
+      // tile down with the group's pairs interleaved -- CTAs working at the same time stream the same
+      // planes and the long tiles start first.  Sub-blocks are numbered through all tiles of this CTA
+      // (g): stream, buffers and barrier phases follow the global number, so the next tile's loads
+      // and first Q K^T run under the current tile's last P V and its epilogue.
       bool ok = true;
-      for (int sb = 0; sb < nsb && ok; ++sb) {
-        const int x = sb & 1;
-        if (sb >= 2) ok = mbar_wait(&bars.v_empty[x], ((sb >> 1) & 1) ^ 1, abort_flag);  // P V(sb-2) done
+      uint32_t g = 0;
+      // The next tile is decoded (request lookup, the tile's last selected position) a few sub-blocks
+      // before the current tile ends, so the lookup's global-memory latency is hidden; the counter
+      // itself is drawn one tile further ahead.
+      for (int n = 0; ok; ++n) {
+        const TileInfo ti = next.ti;
+        const CUtensorMap *map_q = next.map_q, *map_kv = next.map_kv;
+        const int slot = n & 1;
+        if (n >= 2) ok = mbar_wait(&bars.tile_empty[slot], ((n >> 1) & 1) ^ 1, abort_flag);  // tile n-2 has been read
         if (!ok) break;
-        load_v(sb);
-        if (sb + 2 < nsb) {
-          ok = mbar_wait(&bars.k_empty[x], (sb >> 1) & 1, abort_flag);  // S(sb) done
-          if (!ok) break;
-          load_k(sb + 2);
+        s_tiles[slot] = ti;
+        mbar_arrive(&bars.tile_full[slot]);
+        if (ti.nsb == 0) break;
+        const int nsb = ti.nsb, l = ti.l, hk = ti.hk;
+        if (n >= 1) ok = mbar_wait(&bars.q_empty, (n - 1) & 1, abort_flag);  // the previous tile's S MMAs have read Q
+        if (!ok) break;
+        tensormap_acquire(map_q);
+        tensormap_acquire(map_kv);
+        mbar_expect_tx(&bars.q_full, kTileBytes);
+        tma_load_4d(sQ, map_q, 0, hk * rep, ti.i_base, l, &bars.q_full);
+        tma_load_4d(sQ + kHalfBytes, map_q, 64, hk * rep, ti.i_base, l, &bars.q_full);
+        // Loads are issued in the order their buffers come free: K(sb+2) as soon as S(sb) has read
+        // K(sb), V(sb) as soon as P V(sb-2) has read V(sb-2):  K0 K1 | V0 K2 | V1 K3 | ...
+        auto load_k = [&](int sb) {  // false: gave up waiting for the buffer
+          const uint32_t gg = g + sb;
+          const int x = gg & 1;
+          if (gg >= 2 && !mbar_wait(&bars.k_empty[x], ((gg >> 1) & 1) ^ 1, abort_flag)) return false;  // S(gg-2) done
+          mbar_expect_tx(&bars.k_full[x], kSubBytes);
+          tma_load_5d(sK + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
+          tma_load_5d(sK + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
+          return true;
+        };
+        auto load_v = [&](int sb) {
+          const uint32_t gg = g + sb;
+          const int x = gg & 1;
+          if (gg >= 2 && !mbar_wait(&bars.v_empty[x], ((gg >> 1) & 1) ^ 1, abort_flag)) return false;  // P V(gg-2) done
+          mbar_expect_tx(&bars.v_full[x], kSubBytes);
+          tma_load_5d(sV + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
+          tma_load_5d(sV + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 1, l, &bars.v_full[x]);
+          return true;
+        };
+        ok = load_k(0);
+        if (ok && nsb > 1) ok = load_k(1);
+        const int sb_decode = nsb > 4 ? nsb - 4 : 0;  // a few sub-blocks before the tile's end
+        for (int sb = 0; sb < nsb && ok; ++sb) {
+          ok = load_v(sb);
+          if (ok && sb + 2 < nsb) ok = load_k(sb + 2);
+          if (PERSISTENT && ok && sb == sb_decode) next = decode_next();
         }
+        if (!PERSISTENT) next.ti.nsb = 0;  // one tile per CTA
+        g += nsb;
       }
     }
   } else if (warp == 1) {
@@ -344,12 +426,13 @@ __global__ void __launch_bounds__(kThreads, 2)
       const uint32_t idesc_s = instr_desc<DT>(kSubKeys, false);
       const uint32_t idesc_pv = instr_desc<DT>(kD, true);
       const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-      bool ok = mbar_wait(&bars.q_full, 0, abort_flag);
+      bool ok = true;
       // descriptors differ only in their start-address field (units of 16 bytes, low word)
       const uint64_t q_desc = smem_desc(q_addr, 16, 1024);
       const uint64_t k_desc = smem_desc(k_addr, 16, 1024);
       const uint64_t v_desc = smem_desc(v_addr, kSubBytes / 2, 1024);
-      auto issue_s = [&](int sb) {  // S_x = Q K_x^T, N = 64 keys
+      // sb below is the sub-block's number through all tiles of this CTA
+      auto issue_s = [&](uint32_t sb) {  // S_x = Q K_x^T, N = 64 keys
         const int x = sb & 1;
         if (!mbar_wait(&bars.k_full[x], (sb >> 1) & 1, abort_flag)) return false;
         tc_fence_after();
@@ -364,43 +447,81 @@ __global__ void __launch_bounds__(kThreads, 2)
         tc_commit(&bars.k_empty[x]);
         return true;
       };
-      auto issue_pv = [&](int sb) {  // O += P_x V_x, 64 keys = 4 steps of 16
+      auto issue_pv = [&](uint32_t sb, bool first) {  // O (+)= P_x V_x, 64 keys = 4 steps of 16
         const int x = sb & 1;
         const uint32_t ph = (sb >> 1) & 1;
         if (!mbar_wait(&bars.p_full[x], ph, abort_flag) || !mbar_wait(&bars.v_full[x], ph, abort_flag)) return false;
         tc_fence_after();
-#pragma unroll
         const uint64_t vd = v_desc + (uint64_t)(x * (kSubBytes >> 4));
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {  // 16 keys = 2048 bytes of V; the two 64-wide halves of d are 8 KB apart
-          mma_ts(tmem_O, tmem_S + x * kSubKeys + ks * 8, vd + (ks * 2048 >> 4), idesc_pv, (sb > 0 || ks > 0));
+          mma_ts(tmem_O, tmem_S + x * kSubKeys + ks * 8, vd + (ks * 2048 >> 4), idesc_pv, (!first || ks > 0));
         }
         tc_commit(&bars.v_empty[x]);
         return true;
       };
-      if (ok) ok = issue_s(0);
-      if (ok && nsb > 1) ok = issue_s(1);
-      for (int sb = 0; sb < nsb && ok; ++sb) {
-        ok = issue_pv(sb);
-        if (ok && sb + 2 < nsb) ok = issue_s(sb + 2);
+      uint32_t g = 0;
+      for (int n = 0; ok; ++n) {
+        const int slot = n & 1;
+        ok = mbar_wait(&bars.tile_full[slot], (n >> 1) & 1, abort_flag);
+        if (!ok) break;
+        const int nsb = s_tiles[slot].nsb;
+        mbar_arrive(&bars.tile_empty[slot]);
+        if (nsb == 0) break;
+        ok = mbar_wait(&bars.q_full, n & 1, abort_flag);
+        if (!ok) break;
+        // This thread's instruction stream paces the tensor core, so the loops below carry nothing
+        // but the MMAs: first the part of the tile that still has Q K^T to issue, then a commit that
+        // frees Q for the next tile's load, then the last two P V.
+        ok = issue_s(g);
+        if (ok && nsb > 1) ok = issue_s(g + 1);
+        // the first P V of a tile overwrites O: the previous tile's epilogue must have read it
+        if (PERSISTENT && ok && n > 0) {
+          ok = mbar_wait(&bars.o_empty, (n - 1) & 1, abort_flag);
+          tc_fence_after();
+        }
+        int sb = 0;
+        for (; sb + 2 < nsb && ok; ++sb) {
+          ok = issue_pv(g + sb, sb == 0);
+          if (ok) ok = issue_s(g + sb + 2);
+        }
+        if (PERSISTENT && ok) tc_commit(&bars.q_empty);
+        for (; sb < nsb && ok; ++sb) ok = issue_pv(g + sb, sb == 0);
+        if (ok) tc_commit(&bars.o_full);
+        g += nsb;
       }
-      if (ok) tc_commit(&bars.o_full);
     }
   } else {
     // ------------------------------------------------------------------ softmax + epilogue (warps 2..5)
     const int quarter = warp & 3;              // TMEM lanes this warp may touch
     const int row = quarter * 32 + lane;       // row of the tile = TMEM lane
     const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-    const int i_row = i_base + row / rep;
-    const int t_row = i_row < n_sel ? rq.sel[i_row] : -1;
+    bool ok = true;
+    uint32_t g = 0;  // sub-blocks of the tiles before this one
+    for (int n = 0; ok; ++n) {
+    const int slot = n & 1;
+    ok = __all_sync(0xffffffffu, mbar_wait(&bars.tile_full[slot], (n >> 1) & 1, abort_flag));
+    if (!ok) break;
+    // Only what the sub-block loop needs is read now; the slot is released after the epilogue has
+    // read the rest, which keeps registers free in the loop (the producer needs the slot two tiles on).
+    const int nsb = s_tiles[slot].nsb;
+    if (nsb == 0) {
+      mbar_arrive(&bars.tile_empty[slot]);
+      break;
+    }
+    int t_row;
+    {
+      const int i_row = s_tiles[slot].i_base + row / rep;
+      t_row = i_row < s_tiles[slot].n_sel ? s_tiles[slot].sel[i_row] : -1;
+    }
     int warp_tmin = t_row;
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) warp_tmin = min(warp_tmin, __shfl_xor_sync(0xffffffffu, warp_tmin, o));
     float m_ref = -INFINITY, l_sum = 0.f;
-    bool ok = true;
     for (int sb = 0; sb < nsb; ++sb) {
-      const int x = sb & 1;
-      ok = mbar_wait(&bars.s_full[x], (sb >> 1) & 1, abort_flag);
+      const uint32_t gg = g + sb;
+      const int x = gg & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars.s_full[x], (gg >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
       const int key0 = sb * kSubKeys;
@@ -437,8 +558,8 @@ __global__ void __launch_bounds__(kThreads, 2)
       if (rescale) {
         // no P V may be accumulating into O: the previous sub-block's must have completed, and the
         // next one cannot start before this thread has arrived on p_full
-        ok = mbar_wait(&bars.v_empty[(sb - 1) & 1], ((sb - 1) >> 1) & 1, abort_flag);
-        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        ok = __all_sync(0xffffffffu, mbar_wait(&bars.v_empty[(gg - 1) & 1], ((gg - 1) >> 1) & 1, abort_flag));
+        if (!ok) break;
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
@@ -477,30 +598,40 @@ __global__ void __launch_bounds__(kThreads, 2)
       tc_fence_before();
       mbar_arrive(&bars.p_full[x]);
     }
-    // epilogue: O / l -> global
-    if (ok) ok = mbar_wait(&bars.o_full, 0, abort_flag);
-    if (ok) {
-      tc_fence_after();
-      const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-      const int hq = hk * rep + row % rep;
-      uint8_t* orow = rq.out + (((size_t)l * rq.sel_capacity + i_row) * m.Hq + hq) * (kD * 2);
+    if (!ok) break;
+    // epilogue: O / l leaves TMEM as packed 16-bit rows (64 registers); O is then handed back to the
+    // MMA thread, whose next tile's first P V overwrites it, and the rows go out to global memory
+    ok = __all_sync(0xffffffffu, mbar_wait(&bars.o_full, n & 1, abort_flag));
+    if (!ok) break;
+    tc_fence_after();
+    const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
+    const TileInfo ti = s_tiles[slot];
+    mbar_arrive(&bars.tile_empty[slot]);
+    const int i_row = ti.i_base + row / rep;
+    const bool live_row = i_row < ti.n_sel;
+    uint8_t* orow = ti.out + (((size_t)ti.l * ti.sel_capacity + i_row) * m.Hq + ti.hk * rep + row % rep) * (kD * 2);
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld32(tmem_O + lane_addr + c * 32, r);
-        if (i_row < n_sel) {
+    for (int c = 0; c < 4; ++c) {
+      uint32_t r[32];
+      tmem_ld32(tmem_O + lane_addr + c * 32, r);
+      if (c == 3) {  // O has left TMEM: the MMA thread may start the next tile's P V
+        tc_fence_before();
+        mbar_arrive(&bars.o_empty);
+      }
+      if (live_row) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 w;
-            w.x = pack2<DT>(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-            w.y = pack2<DT>(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-            w.z = pack2<DT>(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-            w.w = pack2<DT>(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + (c * 32 + i) * 2) = w;
-          }
+        for (int i = 0; i < 32; i += 8) {
+          uint4 w;
+          w.x = pack2<DT>(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
+          w.y = pack2<DT>(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+          w.z = pack2<DT>(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
+          w.w = pack2<DT>(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+          *reinterpret_cast<uint4*>(orow + (c * 32 + i) * 2) = w;
         }
       }
     }
+    g += nsb;
+    }  // tiles
   }
 
   // ------------------------------------------------------------------ teardown (all roles)
@@ -531,9 +662,13 @@ cudaError_t attention_tc_configure() {
     if (!fn || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
     g_encode = reinterpret_cast<EncodeTiledFn>(fn);
   }
-  cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<KVB_DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_tc_kernel<KVB_DT_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  const void* fns[4] = {(const void*)attn_tc_kernel<KVB_DT_BF16, true>, (const void*)attn_tc_kernel<KVB_DT_BF16, false>,
+                        (const void*)attn_tc_kernel<KVB_DT_F16, true>, (const void*)attn_tc_kernel<KVB_DT_F16, false>};
+  for (const void* f : fns) {
+    cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 // Host: the two tensor maps of one request (Q tile boxes, K/V block boxes), written to `out[0..1]`.
@@ -564,14 +699,24 @@ int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity
 }
 
 cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,
-                                float scale, uint32_t* status, cudaStream_t st) {
-  const unsigned grid = (unsigned)total_tiles * m.Hkv * m.L;
+                                float scale, uint32_t* status, unsigned int* tile_counter, int n_sm, bool persistent,
+                                cudaStream_t st) {
+  const long long work = (long long)total_tiles * m.Hkv * m.L;
   const float scale_log2 = scale * 1.4426950408889634f;
   const CUtensorMap* mp = static_cast<const CUtensorMap*>(maps);
-  if (m.dtype == KVB_DT_BF16)
-    attn_tc_kernel<KVB_DT_BF16><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status);
-  else
-    attn_tc_kernel<KVB_DT_F16><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status);
+  if (persistent) {  // two CTAs per SM; each takes tiles from *tile_counter (zero at launch) until they run out
+    const unsigned grid = (unsigned)(work < 2LL * n_sm ? work : 2LL * n_sm);
+    if (m.dtype == KVB_DT_BF16)
+      attn_tc_kernel<KVB_DT_BF16, true><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+    else
+      attn_tc_kernel<KVB_DT_F16, true><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+  } else {
+    const unsigned grid = (unsigned)work;
+    if (m.dtype == KVB_DT_BF16)
+      attn_tc_kernel<KVB_DT_BF16, false><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+    else
+      attn_tc_kernel<KVB_DT_F16, false><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+  }
   return cudaGetLastError();
 }
 

@@ -35,7 +35,9 @@ struct kvb_ctx {
   int next_slot = 0;
   size_t arena_bytes = 0;
   bool acc_dirty = false;
+  int n_sm = 0;
   bool attn_legacy = false;  // KVB_ATTN=mma selects the warp-level mma.sync kernel (debug aid)
+  int attn_mode = 0;         // KVB_ATTN=onetile (2): one tile per CTA instead of persistent CTAs (cross-check)
   cudaStream_t last_stream = nullptr;
   int64_t launches = 0;
   char err[512] = {0};
@@ -193,6 +195,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   kvb_ctx* c = new (std::nothrow) kvb_ctx();
   if (!c) return KVB_ERR_CUDA;
   c->device = device;
+  c->n_sm = prop.multiProcessorCount;
   c->model = m;
   c->limits = *limits;
   c->dims = ModelDims{m.L, m.Hq, m.Hkv, m.d, m.chunk_tokens, m.kv_dtype, m.int4_group};
@@ -211,6 +214,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, attention_tc_configure());
   const char* attn_env = getenv("KVB_ATTN");
   c->attn_legacy = attn_env && strcmp(attn_env, "mma") == 0;
+  c->attn_mode = attn_env && strcmp(attn_env, "persistent") == 0 ? 1 : (attn_env && strcmp(attn_env, "onetile") == 0 ? 2 : 0);
 
   const int half = m.d / 2;
   std::vector<double> inv(half);
@@ -220,7 +224,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, cudaMalloc(&c->cs_table, (size_t)limits->max_chunks_total * half * sizeof(float2)));
 
   const size_t a1 = sizeof(ChunkDesc) * (size_t)limits->max_chunks_total;
-  const size_t a2 = (sizeof(ReqDesc) + 256) * (size_t)limits->max_requests + 128 + sizeof(SeamWindow) * (size_t)limits->max_chunks_total;
+  const size_t a2 = (sizeof(ReqDesc) + 256) * (size_t)limits->max_requests + 384 + sizeof(SeamWindow) * (size_t)limits->max_chunks_total;
   c->arena_bytes = ((a1 + 255) & ~(size_t)255) + ((a2 + 255) & ~(size_t)255);  // the fused call uploads both tables
   KVB_CUDA(c, cudaMalloc(&c->arena_dev, c->arena_bytes));
   KVB_CUDA(c, cudaMallocHost(&c->staging, c->arena_bytes * kSlots));
@@ -523,14 +527,20 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
       if (e != 0) return fail(c, KVB_ERR_CUDA, "request %d: tensor map encoding failed (%d)", r, e);
     }
   }
-  const int up = upload(c, slot, host, maps_off + 256 * (size_t)n_req, st);
+  const size_t counter_off = maps_off + 256 * (size_t)n_req;  // the attention kernel's tile counter, uploaded as zero
+  memset(host + counter_off, 0, 128);
+  const int up = upload(c, slot, host, counter_off + 128, st);
   if (up != KVB_OK) return up;
   c->last_stream = st;
   const ReqDesc* rd_dev = reinterpret_cast<const ReqDesc*>(c->arena_dev);
+  // persistent CTAs measured faster at every prompt length (most for short prompts, whose tiles are a
+  // few sub-blocks long); KVB_ATTN=onetile selects one tile per CTA (cross-check)
+  const bool persistent = c->attn_mode != 2;
   if (c->attn_legacy)
     KVB_CUDA(c, launch_attention_mma(rd_dev, n_req, tiles, c->dims, softmax_scale, st));
   else
-    KVB_CUDA(c, launch_attention_tc(rd_dev, c->arena_dev + maps_off, n_req, tiles, c->dims, softmax_scale, c->status_dev, st));
+    KVB_CUDA(c, launch_attention_tc(rd_dev, c->arena_dev + maps_off, n_req, tiles, c->dims, softmax_scale, c->status_dev,
+                                    reinterpret_cast<unsigned int*>(c->arena_dev + counter_off), c->n_sm, persistent, st));
   c->launches += 1;
   return KVB_OK;
 }

@@ -85,8 +85,11 @@ cudaError_t attention_mma_configure();
 cudaError_t attention_tc_configure();
 // Encodes the request's two TMA tensor maps (Q, KV) into out[0..255]; returns 0 on success.
 int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity, const void* kv_buf, int T, void* out);
+// persistent: 2 CTAs per SM drawing tiles from *tile_counter (a zeroed device word), else one tile per CTA;
+// n_sm: SMs of the device
 cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,
-                                float scale, uint32_t* status, cudaStream_t st);
+                                float scale, uint32_t* status, unsigned int* tile_counter, int n_sm, bool persistent,
+                                cudaStream_t st);
 
 cudaError_t launch_patch(const ReqDesc* reqs, int n_req, int total_tiles, int rows_per_cta, const ModelDims& m,
                          cudaStream_t st);

@@ -122,6 +122,44 @@ def test_attention_sink_tokens_join_the_selection():
         B.kvb_destroy(ctx)
 
 
+def test_attention_persistent_and_one_tile_ctas_agree(monkeypatch):
+    """The attention kernel runs either as persistent CTAs drawing tiles from a counter (short prompts)
+    or with one tile per CTA (long prompts); KVB_ATTN forces either.  Both must give the same bits, on
+    a batch whose tiles are short, ragged and partly empty (sel_capacity = T > n_sel)."""
+    sh = synth.Shape(L=3, Hq=16, Hkv=2)
+    plans = [synth._request(T, sh.C, [synth.MODE_INT8] * (T // sh.C), [((5 * i) % (T // sh.C)) * sh.C for i in range(T // sh.C)]) for T in (128, 640, 1152, 256)]
+    wl = synth.Workload("modes", 31, sh, plans, synth.SelectPlan(ratio=0.2, seam_before=8, seam_after=8))
+    reqs = prepare(wl)
+    outs = {}
+    for mode in ("persistent", "onetile"):
+        monkeypatch.setenv("KVB_ATTN", mode)
+        ctx = B.create_for_shape(sh, 0, max_requests=len(reqs))
+        try:
+            tbl = run_assemble(ctx, reqs)
+            Ts = [r.plan.T for r in reqs]
+            ks = [B.kvb_select_count(T, 0.2) for T in Ts]
+            sel = B.SelectionTable(Ts, ks, Ts, DEV)  # capacity T: many tiles past n_sel have no rows
+            for r in reqs:
+                r.sel_capacity = r.plan.T
+            B.kvb_deviation_topk(ctx, tbl, 0.2, -1, 8, 8, 3, sel)
+            qs = [torch.randn(sh.L, T, sh.Hq, sh.d, device=DEV, generator=torch.Generator(DEV).manual_seed(T)).to(r.fresh.dtype) for T, r in zip(Ts, reqs)]
+            out = [torch.zeros_like(q) for q in qs]
+            for _ in range(2):  # a second call reuses the context's tile counter slot
+                B.kvb_selective_attn(ctx, tbl, sel, qs, out, 1.0 / math.sqrt(sh.d))
+            B.kvb_last_status(ctx)
+            outs[mode] = out
+            if mode == "persistent":
+                for i, r in enumerate(reqs):
+                    n = int(sel.n_sel[i])
+                    r.q = qs[i]
+                    check_attention(sh, r, sel.sel[i].cpu().numpy()[:n], out[i], None, None)
+                    assert not out[i][:, n:].any()
+        finally:
+            B.kvb_destroy(ctx)
+    for a, b in zip(outs["persistent"], outs["onetile"]):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+
+
 def test_empty_selection_and_wide_overlapping_seam_windows():
     wl = synth.workload(0)
     sh = wl.shape
