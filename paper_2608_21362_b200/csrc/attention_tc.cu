@@ -108,6 +108,20 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same with the accumulate flag fixed to 1 (no register, no setp on a register: the issuing
+// thread's instruction count matters).
+__device__ __forceinline__ void mma_ss_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.eq.b32 p, 0, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.eq.b32 p, 0, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc)
+      : "memory");
+}
 // Load 32 columns of this thread's TMEM lane and wait for them: the wait sits in the same asm
 // statement so that no use of the registers can be scheduled before it.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -221,7 +235,7 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
 }
 
 struct __align__(8) Barriers {
-  uint64_t tile_full[2], tile_empty[2], q_full, q_empty, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2],
+  uint64_t tile_full[2], tile_empty[2], q_full, q_empty, k_full[2], v_full[2], v_empty[2], s_full[2], p_full[2],
       o_full, o_empty;
 };
 
@@ -333,7 +347,6 @@ __global__ void __launch_bounds__(kThreads, 2)
       mbar_init(&bars.tile_full[x], 1);
       mbar_init(&bars.tile_empty[x], 129);  // the MMA thread and the 128 softmax threads
       mbar_init(&bars.k_full[x], 1);
-      mbar_init(&bars.k_empty[x], 1);
       mbar_init(&bars.v_full[x], 1);
       mbar_init(&bars.v_empty[x], 1);
       mbar_init(&bars.s_full[x], 1);
@@ -393,7 +406,7 @@ __global__ void __launch_bounds__(kThreads, 2)
         auto load_k = [&](int sb) {  // false: gave up waiting for the buffer
           const uint32_t gg = g + sb;
           const int x = gg & 1;
-          if (gg >= 2 && !mbar_wait(&bars.k_empty[x], ((gg >> 1) & 1) ^ 1, abort_flag)) return false;  // S(gg-2) done
+          if (gg >= 2 && !mbar_wait(&bars.s_full[x], ((gg >> 1) & 1) ^ 1, abort_flag)) return false;  // S(gg-2) has read K(gg-2)
           mbar_expect_tx(&bars.k_full[x], kSubBytes);
           tma_load_5d(sK + x * kSubBytes, map_kv, 0, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
           tma_load_5d(sK + x * kSubBytes + kSubBytes / 2, map_kv, 64, hk, sb * kSubKeys, 0, l, &bars.k_full[x]);
@@ -441,10 +454,12 @@ __global__ void __launch_bounds__(kThreads, 2)
         for (int ks = 0; ks < 8; ++ks) {  // 16 elements of d per step; 4 steps per 64-element box
           const uint32_t qo = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
           const uint32_t ko = (ks >> 2) * (kSubBytes / 2) + (ks & 3) * 32;
-          mma_ss(tmem_S + x * kSubKeys, q_desc + (qo >> 4), kd + (ko >> 4), idesc_s, ks > 0);
+          if (ks == 0)
+            mma_ss(tmem_S + x * kSubKeys, q_desc + (qo >> 4), kd + (ko >> 4), idesc_s, 0);
+          else
+            mma_ss_acc(tmem_S + x * kSubKeys, q_desc + (qo >> 4), kd + (ko >> 4), idesc_s);
         }
         tc_commit(&bars.s_full[x]);
-        tc_commit(&bars.k_empty[x]);
         return true;
       };
       auto issue_pv = [&](uint32_t sb, bool first) {  // O (+)= P_x V_x, 64 keys = 4 steps of 16
@@ -455,7 +470,10 @@ __global__ void __launch_bounds__(kThreads, 2)
         const uint64_t vd = v_desc + (uint64_t)(x * (kSubBytes >> 4));
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks) {  // 16 keys = 2048 bytes of V; the two 64-wide halves of d are 8 KB apart
-          mma_ts(tmem_O, tmem_S + x * kSubKeys + ks * 8, vd + (ks * 2048 >> 4), idesc_pv, (!first || ks > 0));
+          if (ks == 0)
+            mma_ts(tmem_O, tmem_S + x * kSubKeys, vd, idesc_pv, !first);
+          else
+            mma_ts_acc(tmem_O, tmem_S + x * kSubKeys + ks * 8, vd + (ks * 2048 >> 4), idesc_pv);
         }
         tc_commit(&bars.v_empty[x]);
         return true;
