@@ -291,13 +291,17 @@ __global__ void __launch_bounds__(kThreads, 3)
   // Deviation terms of tokens t and t+1 of this half-warp's head: the stored words are still in
   // registers, the fresh row's matching 2 x 8 bytes per lane come from global memory.
   const uint8_t* fresh_rows = cd.fresh + dst_off * 2;
-  auto dev_pair = [&](int t, const uint2& wl0, const uint2& wh0, const uint2& wl1, const uint2& wh1) {
+  // The fresh words of a pair are fetched one pair ahead of their use (f[0..1]: token t, f[2..3]: t+1),
+  // so the loads' latency is covered by the previous pair's arithmetic.
+  auto load_fresh = [&](int t, uint2 (&f)[4]) {
     const uint8_t* f0 = fresh_rows + (size_t)(t * H + h) * (d * 2) + 8 * ln;
     const uint8_t* f1 = f0 + (size_t)H * (d * 2);
-    const uint2 fl0 = __ldcs(reinterpret_cast<const uint2*>(f0)), fh0 = __ldcs(reinterpret_cast<const uint2*>(f0 + 128));
-    const uint2 fl1 = __ldcs(reinterpret_cast<const uint2*>(f1)), fh1 = __ldcs(reinterpret_cast<const uint2*>(f1 + 128));
-    const uint32_t a0[4] = {wl0.x, wl0.y, wh0.x, wh0.y}, b0[4] = {fl0.x, fl0.y, fh0.x, fh0.y};
-    const uint32_t a1[4] = {wl1.x, wl1.y, wh1.x, wh1.y}, b1[4] = {fl1.x, fl1.y, fh1.x, fh1.y};
+    f[0] = __ldcs(reinterpret_cast<const uint2*>(f0)), f[1] = __ldcs(reinterpret_cast<const uint2*>(f0 + 128));
+    f[2] = __ldcs(reinterpret_cast<const uint2*>(f1)), f[3] = __ldcs(reinterpret_cast<const uint2*>(f1 + 128));
+  };
+  auto dev_pair = [&](int t, const uint2& wl0, const uint2& wh0, const uint2& wl1, const uint2& wh1, const uint2 (&f)[4]) {
+    const uint32_t a0[4] = {wl0.x, wl0.y, wh0.x, wh0.y}, b0[4] = {f[0].x, f[0].y, f[1].x, f[1].y};
+    const uint32_t a1[4] = {wl1.x, wl1.y, wh1.x, wh1.y}, b1[4] = {f[2].x, f[2].y, f[3].x, f[3].y};
     float sa[3], sb[3];
     row_sums4<Pack<OutT>::DT>(a0, b0, sa[0], sa[1], sa[2]);
     row_sums4<Pack<OutT>::DT>(a1, b1, sb[0], sb[1], sb[2]);
@@ -374,13 +378,20 @@ __global__ void __launch_bounds__(kThreads, 3)
       wl = store4(orow + 4 * ln, ol);
       wh = store4(orow + 64 + 4 * ln, oh);
     };
+    uint2 fr[4] = {}, fr_next[4] = {};
+    if (dev_on) load_fresh(t0, fr);
     for (int tt = 0; tt < tok_per; tt += 2) {  // tok_per is even and a pair never straddles a part
       const int t = t0 + tt;
       if (!part_ready(t)) break;
+      if (dev_on && tt + 2 < tok_per) load_fresh(t + 2, fr_next);
       uint2 wl0, wh0, wl1, wh1;
       key_row(t, wl0, wh0);
       key_row(t + 1, wl1, wh1);
-      if (dev_on) dev_pair(t, wl0, wh0, wl1, wh1);
+      if (dev_on) {
+        dev_pair(t, wl0, wh0, wl1, wh1, fr);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) fr[i] = fr_next[i];
+      }
     }
   } else {
     // ------------------------------ values (INT8 / INT4 only; never rotated)
@@ -408,13 +419,20 @@ __global__ void __launch_bounds__(kThreads, 3)
       wl = store4(orow + 4 * ln, ol);
       wh = store4(orow + 64 + 4 * ln, oh);
     };
+    uint2 fr[4] = {}, fr_next[4] = {};
+    if (dev_on) load_fresh(t0, fr);
     for (int tt = 0; tt < tok_per; tt += 2) {
       const int t = t0 + tt;
       if (!part_ready(t)) break;
+      if (dev_on && tt + 2 < tok_per) load_fresh(t + 2, fr_next);
       uint2 wl0, wh0, wl1, wh1;
       value_row(t, wl0, wh0);
       value_row(t + 1, wl1, wh1);
-      if (dev_on) dev_pair(t, wl0, wh0, wl1, wh1);
+      if (dev_on) {
+        dev_pair(t, wl0, wh0, wl1, wh1, fr);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) fr[i] = fr_next[i];
+      }
     }
   }
 
