@@ -197,6 +197,20 @@ int kvb_chunk_importance(kvb_ctx* ctx, const kvb_request* reqs, int n_req, float
 int kvb_quantize_chunk(kvb_ctx* ctx, const void* x, int is_value, int bits, void* codes, void* meta,
                        void* cuda_stream);
 
+/* Position-free cache population for keys: x [L][C][H][d] are the keys of a
+ * chunk encoded at positions orig_pos .. orig_pos+C-1.  Every key is rotated
+ * back by R_theta^(-orig_pos) (Rotary Positional Embeddings, Eq. 3 -- the
+ * inverse of the correction a key "cached at one position and reused at
+ * another" needs) and then quantised as in kvb_quantize_chunk (Eq. 6, per
+ * channel).  The stored chunk is the one a prompt starting at position 0 would
+ * produce: list it in a chunk table with orig_pos = 0 and kvb_assemble applies
+ * the single rotation by new_pos.  The rotation runs in float32 in a fixed
+ * order (u = fma(x, cos, +-(x_partner * sin)), cos and sin from a double
+ * angle), which is what makes the codes reproducible bit for bit.
+ * orig_pos in [0, 2^24); bits: 4 or 8; buffers device, 16-byte aligned. */
+int kvb_quantize_keys_at(kvb_ctx* ctx, const void* x, int orig_pos, int bits, void* codes, void* meta,
+                         void* cuda_stream);
+
 /* Cosine deviation of ONE request for callers that cannot allocate GPU memory:
  * a server that gave the whole GPU to its own block pool at start-up, or a
  * latency-critical thread that may not take the device-wide synchronisation an

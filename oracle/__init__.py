@@ -144,6 +144,16 @@ def rope_rotate(rows, theta: float, delta: float) -> np.ndarray:
     return r
 
 
+def unrotate_keys(rows_bits, dtype: int, theta: float, orig_pos: int) -> np.ndarray:
+    """rows_bits [n,H,d] uint16 -> float64 array of the float32 values R_theta^{-orig_pos} x (the keys of
+    a position-free cache entry, before Eq. 6 is applied)."""
+    r = _c(rows_bits, np.uint16)
+    n, H, d = r.shape
+    out = np.zeros((n, H, d), np.float64)
+    lib().kvo_unrotate_keys_f32(_p(r), C.c_int64(n), H, d, dtype, C.c_double(theta), int(orig_pos), _p(out))
+    return out
+
+
 # ---------------------------------------------------------------- assembly
 def assemble(chunks, L, H, d, T, theta, dtype, int4_group, fresh, want_exact=False):
     """chunks: list of dicts {orig_pos,new_pos,n_tokens,mode,k_codes,v_codes,k_meta,v_meta}

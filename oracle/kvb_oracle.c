@@ -15,6 +15,8 @@
  *   kvo_rope_rotate                   Rotary Positional Embeddings, Eq. 3: the
  *                                     correction R_theta^{delta} that a key cached
  *                                     at one position needs at another
+ *   kvo_unrotate_keys_f32             the same rotation by -orig_pos ahead of Eq. 6
+ *                                     (position-free cache population), in float32
  *   kvo_assemble                      Prompt Assembly (CHUNK_REUSE): cached chunks
  *                                     concatenated in prompt order into the
  *                                     [L,2,T,H,d] KV tensor of the Background section
@@ -258,6 +260,34 @@ void kvo_rope_rotate(double* rows, int64_t n, int H, int d, double theta, double
         double lo = v[j], hi = v[j + half];
         v[j] = lo * c - hi * s;
         v[j + half] = hi * c + lo * s;
+      }
+  }
+}
+
+/* Position-free cache population: the keys of a chunk that was encoded at
+ * positions orig_pos.. are rotated back by R_theta^{-orig_pos} before they are
+ * quantised (Eq. 6), so the stored chunk is the one a prompt starting at
+ * position 0 would produce and re-use at new_pos needs the single rotation
+ * R_theta^{new_pos} (Rotary Positional Embeddings, Eq. 3).  The result feeds a
+ * quantiser whose code decision is taken in float32, so this step is float32
+ * too, with one fixed operation order (cos and sin evaluated in double and
+ * rounded to float32; one rounded product, one fused multiply-add):
+ *   u_lo = fma(x_lo, c, x_hi * s)      u_hi = fma(x_hi, c, -(x_lo * s))
+ * rows: [n][H][d] 16-bit; out: [n][H][d] doubles holding float32 values. */
+void kvo_unrotate_keys_f32(const uint16_t* rows, int64_t n, int H, int d, int dtype, double theta, int orig_pos,
+                           double* out) {
+  int half = d / 2;
+  for (int j = 0; j < half; j++) {
+    double f = pow(theta, -2.0 * (double)j / (double)d);
+    double a = (double)orig_pos * f;
+    float c = (float)cos(a), s = (float)sin(a);
+    for (int64_t t = 0; t < n; t++)
+      for (int h = 0; h < H; h++) {
+        int64_t base = (t * H + h) * d;
+        float lo = (float)load16(rows + base + j, dtype), hi = (float)load16(rows + base + j + half, dtype);
+        float p_hi = hi * s, p_lo = lo * s;
+        out[base + j] = (double)fmaf(lo, c, p_hi);
+        out[base + j + half] = (double)fmaf(hi, c, -p_lo);
       }
   }
 }

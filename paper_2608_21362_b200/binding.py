@@ -100,6 +100,7 @@ def lib():
         L.kvb_assemble_select.argtypes = L.kvb_deviation_topk.argtypes
         L.kvb_selective_attn.argtypes = [vp, C.POINTER(kvb_request), C.c_int, C.POINTER(kvb_selection), C.POINTER(vp), C.POINTER(vp), C.c_float, vp]
         L.kvb_quantize_chunk.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp]
+        L.kvb_quantize_keys_at.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp]
         L.kvb_select_count.argtypes = [C.c_int, C.c_double]
         L.kvb_validate.argtypes = [C.POINTER(kvb_model_desc), C.POINTER(kvb_limits), C.POINTER(kvb_request), C.c_int, C.c_int, C.c_char_p, C.c_size_t]
         L.kvb_last_status.argtypes = [vp]
@@ -262,6 +263,12 @@ def kvb_chunk_importance(ctx, table: RequestTable, importance: List[torch.Tensor
 def kvb_quantize_chunk(ctx, x: torch.Tensor, is_value: bool, bits: int, codes: torch.Tensor, meta: torch.Tensor,
                        stream=None, check: bool = True) -> int:
     st = lib().kvb_quantize_chunk(ctx, x.data_ptr(), int(is_value), bits, codes.data_ptr(), meta.data_ptr(), _stream(stream))
+    return _check(ctx, st) if check else st
+
+
+def kvb_quantize_keys_at(ctx, x: torch.Tensor, orig_pos: int, bits: int, codes: torch.Tensor, meta: torch.Tensor,
+                         stream=None, check: bool = True) -> int:
+    st = lib().kvb_quantize_keys_at(ctx, x.data_ptr(), int(orig_pos), bits, codes.data_ptr(), meta.data_ptr(), _stream(stream))
     return _check(ctx, st) if check else st
 
 

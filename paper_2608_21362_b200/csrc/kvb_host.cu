@@ -623,7 +623,20 @@ int kvb_quantize_chunk(kvb_ctx* c, const void* x, int is_value, int bits, void* 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   KVB_CUDA(c, cudaSetDevice(c->device));
   c->last_stream = st;
-  KVB_CUDA(c, launch_quantize(x, is_value ? 1 : 0, bits, codes, meta, c->dims, st));
+  KVB_CUDA(c, launch_quantize(x, is_value ? 1 : 0, bits, codes, meta, c->dims, 0, 0, nullptr, st));
+  c->launches += 1;
+  return KVB_OK;
+}
+
+int kvb_quantize_keys_at(kvb_ctx* c, const void* x, int orig_pos, int bits, void* codes, void* meta, void* cuda_stream) {
+  if (!c) return KVB_ERR_INVALID_ARG;
+  if (!x || !codes || !meta || (bits != 4 && bits != 8)) return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");
+  if (orig_pos < 0 || orig_pos >= (1 << 24)) return fail(c, KVB_ERR_INVALID_ARG, "orig_pos=%d out of range [0, 2^24)", orig_pos);
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(meta)) return fail(c, KVB_ERR_BAD_TABLE, "quantize buffers must be 16-byte aligned");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+  c->last_stream = st;
+  KVB_CUDA(c, launch_quantize(x, 0, bits, codes, meta, c->dims, 1, orig_pos, c->inv_freq, st));
   c->launches += 1;
   return KVB_OK;
 }

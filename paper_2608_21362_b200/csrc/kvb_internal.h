@@ -95,7 +95,8 @@ cudaError_t launch_patch(const ReqDesc* reqs, int n_req, int total_tiles, int ro
                          cudaStream_t st);
 cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, cudaStream_t st);
 
+// unrotate != 0 (keys only): rotate by R^(-orig_pos) before quantising (inv_freq: [d/2] doubles, device)
 cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
-                            cudaStream_t st);
+                            int unrotate, int orig_pos, const double* inv_freq, cudaStream_t st);
 
 }  // namespace kvb

@@ -24,10 +24,14 @@ __device__ __forceinline__ uint32_t code_of(float v, float mn, float s, float le
   return (uint32_t)c;
 }
 
-// keys: thread = channel (h, j); loops over the tokens of each group
-template <int DT>
+// keys: thread = channel (h, j); loops over the tokens of each group.
+// ROT: the chunk was encoded at positions orig_pos..; every key is first rotated back by
+// R_theta^(-orig_pos) (Rotary Positional Embeddings, Eq. 3), so that the stored chunk is position-free
+// and re-use at new_pos needs the single rotation by new_pos.  cos / sin come from a double-precision
+// angle, the rotation itself is float32 in a fixed order: u = fma(x, c, +-(x_partner * s)).
+template <int DT, bool ROT>
 __global__ void quantize_k_kernel(const uint16_t* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ meta,
-                                  int C, int E, int bits, int group_tokens) {
+                                  int C, int E, int bits, int group_tokens, int orig_pos, const double* __restrict__ inv_freq) {
   const int l = blockIdx.x;
   const int G = C / group_tokens;
   const float levels = (float)((1 << bits) - 1);
@@ -35,10 +39,25 @@ __global__ void quantize_k_kernel(const uint16_t* __restrict__ x, uint8_t* __res
   uint8_t* cl = codes + (size_t)l * C * E * bits / 8;
   float* ml = meta + (size_t)l * G * E * 2;
   for (int c = threadIdx.x; c < E; c += blockDim.x) {  // blockDim.x is even and E is even: c keeps its parity
+    float cs = 1.f, sn = 0.f;
+    int partner = c;
+    if (ROT) {
+      const int j = c & 127;  // channel within the head (d = 128); planes pair j with j + 64
+      double s_d, c_d;
+      sincos((double)orig_pos * inv_freq[j & 63], &s_d, &c_d);
+      cs = (float)c_d;
+      sn = j < 64 ? (float)s_d : -(float)s_d;  // low half: + x_hi * s; high half: - x_lo * s
+      partner = c ^ 64;
+    }
+    auto value = [&](int t) {
+      const float v = load16<DT>(xl + (size_t)t * E + c);
+      if (!ROT) return v;
+      return fmaf(v, cs, __fmul_rn(load16<DT>(xl + (size_t)t * E + partner), sn));
+    };
     for (int g = 0; g < G; ++g) {
       float mn = INFINITY, mx = -INFINITY;
       for (int t = g * group_tokens; t < (g + 1) * group_tokens; ++t) {
-        const float v = load16<DT>(xl + (size_t)t * E + c);
+        const float v = value(t);
         mn = fminf(mn, v);
         mx = fmaxf(mx, v);
       }
@@ -46,7 +65,7 @@ __global__ void quantize_k_kernel(const uint16_t* __restrict__ x, uint8_t* __res
       ml[((size_t)g * E + c) * 2 + 0] = s;
       ml[((size_t)g * E + c) * 2 + 1] = mn;
       for (int t = g * group_tokens; t < (g + 1) * group_tokens; ++t) {
-        const uint32_t q = code_of(load16<DT>(xl + (size_t)t * E + c), mn, s, levels);
+        const uint32_t q = code_of(value(t), mn, s, levels);
         if (bits == 8) {
           cl[(size_t)t * E + c] = (uint8_t)q;
         } else {
@@ -104,17 +123,24 @@ __global__ void quantize_v_kernel(const uint16_t* __restrict__ x, uint8_t* __res
 }  // namespace
 
 cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
-                            cudaStream_t st) {
+                            int unrotate, int orig_pos, const double* inv_freq, cudaStream_t st) {
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   uint8_t* cp = static_cast<uint8_t*>(codes);
   float* mp = static_cast<float*>(meta);
   const int E = m.Hkv * m.d;
   if (!is_value) {
     const int gt = bits == 8 ? m.C : m.int4_group;
-    if (m.dtype == KVB_DT_BF16)
-      quantize_k_kernel<KVB_DT_BF16><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt);
-    else
-      quantize_k_kernel<KVB_DT_F16><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt);
+    if (unrotate) {
+      if (m.dtype == KVB_DT_BF16)
+        quantize_k_kernel<KVB_DT_BF16, true><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, orig_pos, inv_freq);
+      else
+        quantize_k_kernel<KVB_DT_F16, true><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, orig_pos, inv_freq);
+    } else {
+      if (m.dtype == KVB_DT_BF16)
+        quantize_k_kernel<KVB_DT_BF16, false><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, 0, nullptr);
+      else
+        quantize_k_kernel<KVB_DT_F16, false><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, 0, nullptr);
+    }
   } else {
     const int gc = bits == 8 ? m.d : m.int4_group;
     if (m.dtype == KVB_DT_BF16)

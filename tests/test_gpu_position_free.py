@@ -1,0 +1,103 @@
+"""Position-free cache population (kvb_quantize_keys_at): keys rotated back by their original position
+before Eq. 6, so that a cached chunk is listed with orig_pos = 0 and re-used with one rotation."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_21362_b200 import binding as B
+from paper_2608_21362_b200 import synth
+from paper_2608_21362_b200.build import build_library
+
+import helpers
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_library()
+
+
+def _keys(sh, seed):
+    g = torch.Generator().manual_seed(seed)
+    x = torch.randn((sh.L, sh.C, sh.Hkv, sh.d), generator=g) * torch.exp(torch.rand((sh.L, 1, sh.Hkv, sh.d), generator=g) * 3.0 - 1.5)
+    return x.to(sh.torch_dtype)
+
+
+def _quantize_at(ctx, sh, x_dev, pos, bits):
+    L, Cn, H, d = x_dev.shape
+    codes = torch.empty((L, Cn, H, d * bits // 8), dtype=torch.uint8, device=DEV)
+    meta = torch.empty((L, 1 if bits == 8 else Cn // sh.int4_group, H, d, 2), dtype=torch.float32, device=DEV)
+    B.kvb_quantize_keys_at(ctx, x_dev, pos, bits, codes, meta)
+    B.kvb_last_status(ctx)
+    return codes, meta
+
+
+@pytest.mark.parametrize("kv_dtype", ["bf16", "fp16"])
+def test_codes_and_metadata_bit_exact(kv_dtype):
+    sh = synth.Shape(L=2, kv_dtype=kv_dtype)
+    dtc = helpers.dt_code(sh)
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        x = _keys(sh, 5)
+        xb = helpers.bits_of(x)
+        for pos in (0, 128, 4096 * 3 + 128, (1 << 24) - 128):
+            for bits, group in ((8, sh.C), (4, sh.int4_group)):
+                codes, meta = _quantize_at(ctx, sh, x.to(DEV), pos, bits)
+                for l in range(sh.L):
+                    u = oracle.unrotate_keys(xb[l], dtc, sh.theta, pos)
+                    oc, om = oracle.quantize_k(u, bits, group)
+                    assert np.array_equal(codes[l].cpu().numpy(), oc), "codes, pos %d bits %d" % (pos, bits)
+                    assert np.array_equal(meta[l].cpu().numpy(), om), "metadata, pos %d bits %d" % (pos, bits)
+        # position 0 is the plain quantiser
+        qk, _ = B.quantize_fns(ctx, sh)
+        c0, m0 = _quantize_at(ctx, sh, x.to(DEV), 0, 8)
+        c1, m1 = qk(x.to(DEV), 8, sh.C)
+        assert torch.equal(c0, c1) and torch.equal(m0, m1)
+        assert B.kvb_quantize_keys_at(ctx, x.to(DEV), -1, 8, c0, m0, check=False) == B.KVB_ERR_INVALID_ARG
+        assert B.kvb_quantize_keys_at(ctx, x.to(DEV), 0, 5, c0, m0, check=False) == B.KVB_ERR_INVALID_ARG
+    finally:
+        B.kvb_destroy(ctx)
+
+
+def test_reuse_at_another_position_is_one_rotation():
+    """Keys encoded at position 896, stored position-free, re-used at position 256: the stitched rows are
+    the original keys rotated by 256 - 896, up to the quantisation step (Eq. 6: half a step per channel,
+    a rotation mixes two channels)."""
+    sh = synth.Shape(L=2)
+    dtc = helpers.dt_code(sh)
+    orig, new, T = 896, 256, 512
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        x = _keys(sh, 9)
+        vals = _keys(sh, 10)
+        codes, meta = _quantize_at(ctx, sh, x.to(DEV), orig, 8)
+        qk, qv = B.quantize_fns(ctx, sh)
+        vcodes, vmeta = qv(vals.to(DEV), 8, sh.d)
+        plan = synth._request(T, sh.C, [synth.MODE_FRESH, synth.MODE_FRESH, synth.MODE_INT8, synth.MODE_FRESH], [0, 0, 0, 0])
+        assert plan.chunks[2].new_pos == new and plan.chunks[2].orig_pos == 0
+
+        class R:
+            pass
+
+        r = R()
+        r.plan = plan
+        r.chunks = [synth.Chunk(c) for c in plan.chunks]
+        r.chunks[2] = synth.Chunk(plan.chunks[2], codes, vcodes, meta, vmeta)
+        r.fresh = torch.zeros((sh.L, 2, T, sh.Hkv, sh.d), dtype=sh.torch_dtype, device=DEV)
+        r.kv_buf = torch.zeros_like(r.fresh)
+        B.kvb_assemble(ctx, B.RequestTable([r]))
+        B.kvb_last_status(ctx)
+        got = oracle.bits_to_f64(helpers.bits_of(r.kv_buf[:, 0, new : new + sh.C]), dtc)  # [L,C,H,d]
+        x64 = oracle.bits_to_f64(helpers.bits_of(x), dtc)
+        half = sh.d // 2
+        for l in range(sh.L):
+            want = oracle.rope_rotate(x64[l], sh.theta, float(new - orig))
+            scale = meta[l, 0].cpu().numpy()[..., 0].astype(np.float64)  # [H,d] step of each stored channel
+            step_pair = np.sqrt(scale[:, :half] ** 2 + scale[:, half:] ** 2)
+            bound = 0.5 * np.concatenate([step_pair, step_pair], -1)[None] * 1.01 + 2.0**-8 * np.abs(want) + 1e-6
+            assert np.all(np.abs(got[l] - want) <= bound)
+    finally:
+        B.kvb_destroy(ctx)

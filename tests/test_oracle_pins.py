@@ -466,3 +466,27 @@ def test_importance_is_the_mean_key_norm():
     assert np.array_equal(oracle.importance(kv2, C, 1), oracle.importance(kv, C, 1))
     dbl = oracle.round_to_bits(oracle.bits_to_f64(kv, 1) * 2.0, 1)
     assert np.allclose(oracle.importance(dbl, C, 1), 2 * oracle.importance(kv, C, 1), rtol=1e-15)
+
+
+# ------------------------------------------------------------------ position-free cache population (rotation by -orig_pos)
+def test_unrotate_keys_is_the_inverse_rotation_in_float32():
+    theta, H, d = 1e6, 2, 16
+    bits = _rand_bits((5, H, d), 1, scale=3.0)
+    x = oracle.bits_to_f64(bits, 1)
+    assert np.array_equal(oracle.unrotate_keys(bits, 1, theta, 0), x)  # position 0: nothing to undo
+    for pos in (1, 50, 1000, 123456, (1 << 24) - 128):
+        u = oracle.unrotate_keys(bits, 1, theta, pos)
+        assert np.array_equal(u, u.astype(np.float32).astype(np.float64))  # float32 values
+        # the pinned forward rotation brings the keys back, up to float32 rounding of a pair
+        back = oracle.rope_rotate(u, theta, float(pos))
+        pair = np.sqrt(x[..., : d // 2] ** 2 + x[..., d // 2 :] ** 2)
+        bound = 4 * 2.0**-24 * np.concatenate([pair, pair], -1) + 1e-30
+        assert np.all(np.abs(back - x) <= bound)
+        # and it is the plain inverse rotation evaluated exactly, to the same bound
+        assert np.all(np.abs(u - oracle.rope_rotate(x, theta, -float(pos))) <= bound)
+    # closed form on unit vectors: plane 0 has frequency 1, so e_0 -> (cos p, -sin p) on (0, d/2)
+    e = np.zeros((1, 1, d))
+    e[0, 0, 0] = 1.0
+    u = oracle.unrotate_keys(oracle.round_to_bits(e, 1), 1, theta, 1000)[0, 0]
+    assert u[0] == np.float32(math.cos(1000.0)) and u[d // 2] == -np.float32(math.sin(1000.0))
+    assert np.all(u[1 : d // 2] == 0) and np.all(u[d // 2 + 1 :] == 0)
