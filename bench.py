@@ -105,10 +105,13 @@ def physical_gpu_index(local: int) -> int:
 class Replica:
     """One independent copy of the workload's requests on the device, with its marshalled tables."""
 
-    def __init__(self, B, ctx, wl, dev, seed_shift):
+    def __init__(self, B, ctx, wl, dev, seed_shift, meta_fp16=False):
         wl = synth.Workload(wl.name, wl.seed + 7919 * seed_shift, wl.shape, wl.requests, wl.select, wl.sigma_bulk, wl.sigma_seam, wl.seam_tokens)
-        qk, qv = B.quantize_fns(ctx, wl.shape)
+        qk, qv = B.quantize_fns(ctx, wl.shape, meta_fp16)
         self.reqs = synth.materialize(wl, dev, qk, qv, B.assemble_fn(ctx))
+        for r in self.reqs:
+            for ck in r.chunks:
+                ck.meta_fp16 = int(ck.k_meta is not None and ck.k_meta.dtype == torch.float16)
         self._pack_payload(dev)
         sp = wl.select
         for r in self.reqs:
@@ -267,6 +270,7 @@ def main():
     ap.add_argument("--replicas", type=int, default=0, help="independent copies rotated through (0 = auto)")
     ap.add_argument("--batch", type=int, default=1, help="requests per step: the workload's request list repeated this many times")
     ap.add_argument("--path", default="one-pass", choices=["one-pass", "two-call"], help="kvb_assemble_select, or kvb_assemble + kvb_deviation_topk")
+    ap.add_argument("--meta-fp16", action="store_true", help="cached chunks carry compact (binary16) scale/min pairs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -308,7 +312,7 @@ def main():
     ctx = B.create_for_shape(sh, local, max_requests=len(wl.requests), max_chunks_total=n_chunks, max_tokens_total=n_tok)
 
     n_rep = args.replicas or {"cfg1": 8, "cfg2": 3, "cfg4": 1}[args.workload]
-    reps = [Replica(B, ctx, wl, dev, 100 * rank + i) for i in range(n_rep)]
+    reps = [Replica(B, ctx, wl, dev, 100 * rank + i, args.meta_fp16) for i in range(n_rep)]
     torch.cuda.synchronize()
     footprint = sum(r.device_bytes() for r in reps)
 
@@ -400,7 +404,8 @@ def main():
     sampler.stop()
 
     # ---- algorithmic work per step
-    asm_bytes = sum(synth.assemble_bytes(sh, r.plan) for r in reps[0].reqs)
+    pair_bytes = 4 if args.meta_fp16 else 8
+    asm_bytes = sum(synth.assemble_bytes(sh, r.plan, pair_bytes) for r in reps[0].reqs)
     dev_bytes = sum(synth.deviation_bytes(sh, r.plan, sp.which) for r in reps[0].reqs)
     flops = []
     for rep in reps:
@@ -424,7 +429,7 @@ def main():
     tensor_peak = peaks["bf16_sustained"] if long_run else peaks["bf16_burst"]
     attn_stage = {"bound": "tensor", "ms": stage_ms[2], "achieved": attn_flops / stage_ms[2] / 1e9, "peak": tensor_peak, "unit": "TFLOP/s", "algorithmic_flops": attn_flops}
     if ONE_PASS:  # stitch + deviation sums + selection behind one call
-        one_bytes = sum(synth.one_pass_bytes(sh, r.plan, sp.which) for r in reps[0].reqs)
+        one_bytes = sum(synth.one_pass_bytes(sh, r.plan, sp.which, pair_bytes) for r in reps[0].reqs)
         ms01 = stage_ms[0] + stage_ms[1]
         stages = {
             "assemble_select": {"bound": "hbm", "ms": ms01, "achieved": one_bytes / ms01 / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s", "algorithmic_bytes": one_bytes,
@@ -457,6 +462,7 @@ def main():
         "dtype": "bf16" if sh.kv_dtype == "bf16" else "fp16", "data": "synthetic",
         "config": {
             "workload": wl.name, "path": "kvb_assemble_select + kvb_selective_attn" if ONE_PASS else "kvb_assemble + kvb_deviation_topk + kvb_selective_attn",
+            "metadata": "binary16 (scale, min) pairs" if args.meta_fp16 else "float32 (scale, min) pairs",
             "requests_per_step": len(wl.requests), "tokens_per_step": n_tok, "layers": sh.L, "q_heads": sh.Hq,
             "kv_heads": sh.Hkv, "head_dim": sh.d, "chunk_tokens": sh.C, "select_ratio": sp.ratio, "seam_window": [sp.seam_before, sp.seam_after],
             "parallelism": "replicas only (one independent stream of requests per GPU)" if world > 1 else "single GPU",

@@ -31,6 +31,10 @@
  *                             chunk), C/int4_group for INT4
  *   value metadata            [L][C][H][G_v][2] float32 (scale, min); statistics per token
  *                             over a channel group: G_v = 1 for INT8, d/int4_group for INT4
+ *   compact metadata          the same two layouts with IEEE binary16 (scale, min) pairs
+ *                             (4 bytes per pair), chunk flag meta_fp16 = 1: min rounded
+ *                             down and scale rounded up to binary16 when the chunk is
+ *                             quantised, codes taken against the rounded pair
  * Cached keys are stored already rotated (RoPE) at absolute positions
  * orig_pos .. orig_pos+C-1, as a prefill pass leaves them.
  */
@@ -80,7 +84,7 @@ typedef struct {
   int32_t n_tokens;         /* must equal the model's chunk_tokens */
   int32_t mode;             /* kvb_mode */
   int32_t match;            /* kvb_match; EXACT requires orig_pos == new_pos */
-  int32_t reserved;
+  int32_t meta_fp16;        /* 0: float32 (scale, min) pairs; 1: binary16 pairs (INT8 / INT4 chunks) */
   const void* k_codes;      /* device; NULL for FRESH */
   const void* v_codes;      /* device; NULL for FRESH */
   const void* k_meta;       /* device; INT8 / INT4 only */
@@ -210,6 +214,17 @@ int kvb_quantize_chunk(kvb_ctx* ctx, const void* x, int is_value, int bits, void
  * orig_pos in [0, 2^24); bits: 4 or 8; buffers device, 16-byte aligned. */
 int kvb_quantize_keys_at(kvb_ctx* ctx, const void* x, int orig_pos, int bits, void* codes, void* meta,
                          void* cuda_stream);
+
+/* The general form of the two calls above.  unrotate_from < 0: no rotation
+ * (kvb_quantize_chunk); >= 0: keys only, rotated back from that position
+ * (kvb_quantize_keys_at).  meta_fp16 = 1 writes compact metadata: per group,
+ * min is rounded down and scale = (max - min_rounded)/(2^b - 1) is rounded up
+ * to binary16 (so every value still falls inside the code range), and the
+ * codes are rint((x - min16)/scale16) in float32 against those rounded values;
+ * the chunk's statistics must lie in binary16's finite range (|x| < 65504,
+ * scale >= 2^-24).  List such a chunk with kvb_chunk.meta_fp16 = 1. */
+int kvb_quantize_chunk_ex(kvb_ctx* ctx, const void* x, int is_value, int bits, int unrotate_from, int meta_fp16,
+                          void* codes, void* meta, void* cuda_stream);
 
 /* Cosine deviation of ONE request for callers that cannot allocate GPU memory:
  * a server that gave the whole GPU to its own block pool at start-up, or a

@@ -97,23 +97,24 @@ def bits_to_f64(b, dtype: int) -> np.ndarray:
 
 
 # ---------------------------------------------------------------- Eq. 6
-def quantize_k(x, bits: int, group_tokens: int):
-    """x [C,H,d] float64 -> (codes u8 [C,H,d] or [C,H,d/2], meta f32 [C/group,H,d,2])."""
+def quantize_k(x, bits: int, group_tokens: int, meta16: bool = False):
+    """x [C,H,d] float64 -> (codes u8 [C,H,d] or [C,H,d/2], meta f32 [C/group,H,d,2]).
+    meta16: compact metadata (min rounded down, scale rounded up to binary16; returned as float32)."""
     x = _c(x, np.float64)
     Cn, H, d = x.shape
     codes = np.zeros((Cn, H, d * bits // 8), np.uint8)
     meta = np.zeros((Cn // group_tokens, H, d, 2), np.float32)
-    lib().kvo_quantize_k(_p(x), Cn, H, d, bits, group_tokens, _p(codes), _p(meta))
+    lib().kvo_quantize_k_ex(_p(x), Cn, H, d, bits, group_tokens, int(meta16), _p(codes), _p(meta))
     return codes, meta
 
 
-def quantize_v(x, bits: int, group_ch: int):
+def quantize_v(x, bits: int, group_ch: int, meta16: bool = False):
     """x [C,H,d] float64 -> (codes, meta f32 [C,H,d/group,2])."""
     x = _c(x, np.float64)
     Cn, H, d = x.shape
     codes = np.zeros((Cn, H, d * bits // 8), np.uint8)
     meta = np.zeros((Cn, H, d // group_ch, 2), np.float32)
-    lib().kvo_quantize_v(_p(x), Cn, H, d, bits, group_ch, _p(codes), _p(meta))
+    lib().kvo_quantize_v_ex(_p(x), Cn, H, d, bits, group_ch, int(meta16), _p(codes), _p(meta))
     return codes, meta
 
 

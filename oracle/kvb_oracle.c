@@ -136,7 +136,22 @@ void kvo_decode_array(const uint16_t* x, int64_t n, int dtype, double* out) {
  * (subtract, divide, round-half-even, clamp) so that a float32 quantiser on
  * any IEEE machine takes the same decisions.  A group with max == min gets
  * scale 1 and all-zero codes, so it dequantises to min exactly. */
-static void quantize_group(const double* x, int n, int64_t stride, int bits, uint8_t* q /* n codes */,
+/* Largest binary16 value <= x (up = 0) or smallest one >= x (up = 1); x finite, inside binary16's range. */
+static float f16_directed(float x, int up) {
+  if (x == 0.0f) return x;
+  int e;
+  (void)frexp(fabs((double)x), &e);
+  int ex = e - 1;
+  if (ex < -14) ex = -14;
+  double quantum = ldexp(1.0, ex - 10);
+  double q = (double)x / quantum; /* exact: a power-of-two scaling */
+  return (float)((up ? ceil(q) : floor(q)) * quantum);
+}
+
+/* meta16: compact metadata -- the minimum is rounded DOWN to binary16, the scale is taken against
+ * the rounded minimum and rounded UP to binary16 (so that no value leaves the code range), and the
+ * codes are decided against that rounded pair. */
+static void quantize_group(const double* x, int n, int64_t stride, int bits, int meta16, uint8_t* q /* n codes */,
                            float* scale_out, float* min_out) {
   float mn = (float)x[0], mx = (float)x[0];
   for (int i = 1; i < n; i++) {
@@ -145,7 +160,9 @@ static void quantize_group(const double* x, int n, int64_t stride, int bits, uin
     if (v > mx) mx = v;
   }
   float levels = (float)((1 << bits) - 1);
+  if (meta16) mn = f16_directed(mn, 0);
   float s = (mx > mn) ? (mx - mn) / levels : 1.0f;
+  if (meta16) s = f16_directed(s, 1);
   for (int i = 0; i < n; i++) {
     float v = (float)x[i * stride];
     float c = rintf((v - mn) / s);
@@ -181,8 +198,8 @@ static int get_code(const uint8_t* codes, int bits, int64_t elem) {
  *   x     [C][H][d] doubles (the cached, already-rotated keys of one layer)
  *   codes [C][H][d] u8, or [C][H][d/2] packed nibbles
  *   meta  [C/group_tokens][H][d][2] float32 (scale, min) */
-void kvo_quantize_k(const double* x, int C, int H, int d, int bits, int group_tokens, uint8_t* codes,
-                    float* meta) {
+void kvo_quantize_k_ex(const double* x, int C, int H, int d, int bits, int group_tokens, int meta16, uint8_t* codes,
+                       float* meta) {
   int G = C / group_tokens;
   uint8_t* tmp = (uint8_t*)malloc((size_t)group_tokens);
   if (bits == 4) memset(codes, 0, (size_t)C * H * d / 2);
@@ -191,7 +208,7 @@ void kvo_quantize_k(const double* x, int C, int H, int d, int bits, int group_to
       for (int j = 0; j < d; j++) {
         const double* base = x + ((int64_t)(g * group_tokens) * H + h) * d + j;
         float* m = meta + (((int64_t)g * H + h) * d + j) * 2;
-        quantize_group(base, group_tokens, (int64_t)H * d, bits, tmp, &m[0], &m[1]);
+        quantize_group(base, group_tokens, (int64_t)H * d, bits, meta16, tmp, &m[0], &m[1]);
         for (int i = 0; i < group_tokens; i++)
           put_code(codes, bits, ((int64_t)(g * group_tokens + i) * H + h) * d + j, tmp[i]);
       }
@@ -201,8 +218,8 @@ void kvo_quantize_k(const double* x, int C, int H, int d, int bits, int group_to
 /* Values, per token: for each (token t, head h) the statistics run over the
  * channels of one group (group_ch consecutive channels).
  *   meta [C][H][d/group_ch][2] float32 (scale, min) */
-void kvo_quantize_v(const double* x, int C, int H, int d, int bits, int group_ch, uint8_t* codes,
-                    float* meta) {
+void kvo_quantize_v_ex(const double* x, int C, int H, int d, int bits, int group_ch, int meta16, uint8_t* codes,
+                       float* meta) {
   int G = d / group_ch;
   uint8_t* tmp = (uint8_t*)malloc((size_t)group_ch);
   if (bits == 4) memset(codes, 0, (size_t)C * H * d / 2);
@@ -211,10 +228,17 @@ void kvo_quantize_v(const double* x, int C, int H, int d, int bits, int group_ch
       for (int g = 0; g < G; g++) {
         int64_t e0 = ((int64_t)t * H + h) * d + g * group_ch;
         float* m = meta + (((int64_t)t * H + h) * G + g) * 2;
-        quantize_group(x + e0, group_ch, 1, bits, tmp, &m[0], &m[1]);
+        quantize_group(x + e0, group_ch, 1, bits, meta16, tmp, &m[0], &m[1]);
         for (int i = 0; i < group_ch; i++) put_code(codes, bits, e0 + i, tmp[i]);
       }
   free(tmp);
+}
+
+void kvo_quantize_k(const double* x, int C, int H, int d, int bits, int group_tokens, uint8_t* codes, float* meta) {
+  kvo_quantize_k_ex(x, C, H, d, bits, group_tokens, 0, codes, meta);
+}
+void kvo_quantize_v(const double* x, int C, int H, int d, int bits, int group_ch, uint8_t* codes, float* meta) {
+  kvo_quantize_v_ex(x, C, H, d, bits, group_ch, 0, codes, meta);
 }
 
 /* Inverse of Eq. 6:  x^ = q * scale + min, in double. */

@@ -32,7 +32,7 @@ class kvb_chunk(C.Structure):
         ("n_tokens", C.c_int32),
         ("mode", C.c_int32),
         ("match", C.c_int32),
-        ("reserved", C.c_int32),
+        ("meta_fp16", C.c_int32),
         ("k_codes", C.c_void_p),
         ("v_codes", C.c_void_p),
         ("k_meta", C.c_void_p),
@@ -101,6 +101,7 @@ def lib():
         L.kvb_selective_attn.argtypes = [vp, C.POINTER(kvb_request), C.c_int, C.POINTER(kvb_selection), C.POINTER(vp), C.POINTER(vp), C.c_float, vp]
         L.kvb_quantize_chunk.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp]
         L.kvb_quantize_keys_at.argtypes = [vp, vp, C.c_int, C.c_int, vp, vp, vp]
+        L.kvb_quantize_chunk_ex.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
         L.kvb_select_count.argtypes = [C.c_int, C.c_double]
         L.kvb_validate.argtypes = [C.POINTER(kvb_model_desc), C.POINTER(kvb_limits), C.POINTER(kvb_request), C.c_int, C.c_int, C.c_char_p, C.c_size_t]
         L.kvb_last_status.argtypes = [vp]
@@ -133,6 +134,7 @@ class RequestTable:
                 chunks[i].orig_pos, chunks[i].new_pos = p.orig_pos, p.new_pos
                 chunks[i].n_tokens = chunk_tokens
                 chunks[i].mode, chunks[i].match = p.mode, p.match
+                chunks[i].meta_fp16 = int(getattr(ck, "meta_fp16", 0))
                 for name in ("k_codes", "v_codes", "k_meta", "v_meta"):
                     t = getattr(ck, name)
                     if t is not None:
@@ -272,6 +274,13 @@ def kvb_quantize_keys_at(ctx, x: torch.Tensor, orig_pos: int, bits: int, codes: 
     return _check(ctx, st) if check else st
 
 
+def kvb_quantize_chunk_ex(ctx, x: torch.Tensor, is_value: bool, bits: int, unrotate_from: int, meta_fp16: bool,
+                          codes: torch.Tensor, meta: torch.Tensor, stream=None, check: bool = True) -> int:
+    st = lib().kvb_quantize_chunk_ex(ctx, x.data_ptr(), int(is_value), bits, int(unrotate_from), int(meta_fp16),
+                                     codes.data_ptr(), meta.data_ptr(), _stream(stream))
+    return _check(ctx, st) if check else st
+
+
 def kvb_deviation_static(device: int, model: kvb_model_desc, kv_buf: torch.Tensor, fresh: torch.Tensor, T: int,
                          which: int, delta: torch.Tensor, stream=None) -> int:
     """Deviation of one request without a context and without any allocation (static device scratch,
@@ -299,18 +308,20 @@ def create_for_shape(sh, device: int = 0, max_requests: int = 64, max_chunks_tot
                       max_chunks_total, max_tokens_total)
 
 
-def quantize_fns(ctx, sh):
-    """(quantize_k, quantize_v) callables in the form synth.materialize expects, running the CUDA quantiser."""
+def quantize_fns(ctx, sh, meta_fp16: bool = False):
+    """(quantize_k, quantize_v) callables in the form synth.materialize expects, running the CUDA quantiser.
+    meta_fp16: compact metadata (torch.float16 pairs; mark the chunk with meta_fp16 = 1)."""
+    mt = torch.float16 if meta_fp16 else torch.float32
 
     def _q(x: torch.Tensor, bits: int, is_value: bool):
         L, Cn, H, d = x.shape
         x = x.contiguous()
         codes = torch.empty((L, Cn, H, d * bits // 8), dtype=torch.uint8, device=x.device)
         if is_value:
-            meta = torch.empty((L, Cn, H, 1 if bits == 8 else d // sh.int4_group, 2), dtype=torch.float32, device=x.device)
+            meta = torch.empty((L, Cn, H, 1 if bits == 8 else d // sh.int4_group, 2), dtype=mt, device=x.device)
         else:
-            meta = torch.empty((L, 1 if bits == 8 else Cn // sh.int4_group, H, d, 2), dtype=torch.float32, device=x.device)
-        kvb_quantize_chunk(ctx, x, is_value, bits, codes, meta)
+            meta = torch.empty((L, 1 if bits == 8 else Cn // sh.int4_group, H, d, 2), dtype=mt, device=x.device)
+        kvb_quantize_chunk_ex(ctx, x, is_value, bits, -1, meta_fp16, codes, meta)
         return codes, meta
 
     return (lambda x, bits, group: _q(x, bits, False)), (lambda x, bits, group: _q(x, bits, True))

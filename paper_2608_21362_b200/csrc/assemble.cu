@@ -205,16 +205,18 @@ __global__ void __launch_bounds__(kThreads, 3)
   int G = 1;        // value channel groups per row
   int g_first = 0;  // first key token group held in shared memory
   const int group_tokens = bits == 8 ? m.C : m.int4_group;
+  const bool meta16 = cd.meta16 != 0;      // (scale, min) pairs of 2 x 2 bytes instead of 2 x 4
+  const uint32_t pair_bytes = meta16 ? 4 : 8;
   if (bits != 16) {
     if (!kv) {
       const int G_layer = m.C / group_tokens;
       g_first = tb / group_tokens;
       const int n_g = (tb + C - 1) / group_tokens - g_first + 1;
-      meta_bytes = (uint32_t)(n_g * row_elems * 8);
-      meta_g = reinterpret_cast<const uint8_t*>(cd.k_meta) + ((size_t)l * G_layer + g_first) * row_elems * 8;
+      meta_bytes = (uint32_t)(n_g * row_elems * pair_bytes);
+      meta_g = reinterpret_cast<const uint8_t*>(cd.k_meta) + ((size_t)l * G_layer + g_first) * row_elems * pair_bytes;
     } else {
       G = bits == 8 ? 1 : d / m.int4_group;
-      meta_bytes = (uint32_t)(C * H * G * 8);
+      meta_bytes = (uint32_t)(C * H * G * pair_bytes);
       meta_g = reinterpret_cast<const uint8_t*>(cd.v_meta) + ((size_t)l * split + part_id) * meta_bytes;
     }
   }
@@ -344,11 +346,25 @@ __global__ void __launch_bounds__(kThreads, 3)
         const int g = (tb + t) / group_tokens - g_first;
         if (g != cur_group) {
           cur_group = g;
-          const float* mlo = s_meta + ((size_t)(g * H + h) * d + 4 * ln) * 2;
-          const float4 a0 = *reinterpret_cast<const float4*>(mlo), a1 = *reinterpret_cast<const float4*>(mlo + 4);
-          const float4 b0 = *reinterpret_cast<const float4*>(mlo + 128), b1 = *reinterpret_cast<const float4*>(mlo + 132);
-          const float sl[4] = {a0.x, a0.z, a1.x, a1.z}, ml[4] = {a0.y, a0.w, a1.y, a1.w};
-          const float sh[4] = {b0.x, b0.z, b1.x, b1.z}, mh[4] = {b0.y, b0.w, b1.y, b1.w};
+          float sl[4], ml[4], sh[4], mh[4];  // (scale, min) of this lane's 4 low and 4 high channels
+          const size_t pair = (size_t)(g * H + h) * d + 4 * ln;
+          if (meta16) {
+            const uint4 a = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(s_meta) + pair * 4);
+            const uint4 b = *reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(s_meta) + (pair + 64) * 4);
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 lo = __half22float2(*reinterpret_cast<const __half2*>(&aw[i]));
+              const float2 hi = __half22float2(*reinterpret_cast<const __half2*>(&bw[i]));
+              sl[i] = lo.x, ml[i] = lo.y, sh[i] = hi.x, mh[i] = hi.y;
+            }
+          } else {
+            const float* mlo = s_meta + pair * 2;
+            const float4 a0 = *reinterpret_cast<const float4*>(mlo), a1 = *reinterpret_cast<const float4*>(mlo + 4);
+            const float4 b0 = *reinterpret_cast<const float4*>(mlo + 128), b1 = *reinterpret_cast<const float4*>(mlo + 132);
+            sl[0] = a0.x, sl[1] = a0.z, sl[2] = a1.x, sl[3] = a1.z, ml[0] = a0.y, ml[1] = a0.w, ml[2] = a1.y, ml[3] = a1.w;
+            sh[0] = b0.x, sh[1] = b0.z, sh[2] = b1.x, sh[3] = b1.z, mh[0] = b0.y, mh[1] = b0.w, mh[2] = b1.y, mh[3] = b1.w;
+          }
           float al[4], bl[4], cl[4], ah[4], bh[4], ch[4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
@@ -399,13 +415,17 @@ __global__ void __launch_bounds__(kThreads, 3)
       const int u = t * H + h;
       OutT* orow = dst + (size_t)u * d;
       float s_lo, m_lo, s_hi, m_hi;
+      auto pair_at = [&](size_t pair) {  // (scale, min) pair number `pair` of the staged metadata
+        if (meta16) return __half22float2(reinterpret_cast<const __half2*>(s_meta)[pair]);
+        return *reinterpret_cast<const float2*>(s_meta + pair * 2);
+      };
       if (bits == 8) {
-        const float2 sm = *reinterpret_cast<const float2*>(s_meta + (size_t)u * 2);
+        const float2 sm = pair_at((size_t)u);
         s_lo = s_hi = sm.x, m_lo = m_hi = sm.y;
       } else {
         const int g_lo = (4 * ln) / m.int4_group, g_hi = (64 + 4 * ln) / m.int4_group;
-        const float2 a = *reinterpret_cast<const float2*>(s_meta + ((size_t)u * G + g_lo) * 2);
-        const float2 b = *reinterpret_cast<const float2*>(s_meta + ((size_t)u * G + g_hi) * 2);
+        const float2 a = pair_at((size_t)u * G + g_lo);
+        const float2 b = pair_at((size_t)u * G + g_hi);
         s_lo = a.x, m_lo = fmaf(-bias, a.x, a.y), s_hi = b.x, m_hi = fmaf(-bias, b.x, b.y);
       }
       uint64_t ql[2], qh[2], ol[2], oh[2];

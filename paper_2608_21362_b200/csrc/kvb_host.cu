@@ -98,6 +98,7 @@ int check_request(kvb_ctx* c, const kvb_request& r, int ri, bool need_payload) {
     if (k.new_pos != i * C)
       return fail(c, KVB_ERR_BAD_TABLE, "request %d chunk %d: new_pos=%d leaves a gap or overlap (expected %d)", ri, i, k.new_pos, i * C);
     if (k.mode < KVB_MODE_FRESH || k.mode > KVB_MODE_INT4) return fail(c, KVB_ERR_INVALID_ARG, "request %d chunk %d: bad mode %d", ri, i, k.mode);
+    if (k.meta_fp16 != 0 && k.meta_fp16 != 1) return fail(c, KVB_ERR_INVALID_ARG, "request %d chunk %d: bad meta_fp16 %d", ri, i, k.meta_fp16);
     if (k.match < KVB_MATCH_MISS || k.match > KVB_MATCH_APPROX) return fail(c, KVB_ERR_INVALID_ARG, "request %d chunk %d: bad match %d", ri, i, k.match);
     if (k.mode == KVB_MODE_FRESH) continue;
     if (k.orig_pos < 0 || k.orig_pos >= (1 << 24) || k.new_pos >= (1 << 24))
@@ -286,6 +287,7 @@ size_t pack_chunks(kvb_ctx* c, const kvb_request* reqs, int n_req, ChunkDesc* cd
       d.delta_pos = k.mode == KVB_MODE_FRESH ? 0 : k.new_pos - k.orig_pos;
       d.mode = k.mode;
       d.tok_offset = tok;
+      d.meta16 = k.meta_fp16;
       cd[n] = d;
       const size_t s = assemble_smem_bytes(c->dims, k.mode);
       if (s > smem) smem = s;
@@ -616,29 +618,30 @@ int kvb_chunk_importance(kvb_ctx* c, const kvb_request* reqs, int n_req, float* 
   return KVB_OK;
 }
 
-int kvb_quantize_chunk(kvb_ctx* c, const void* x, int is_value, int bits, void* codes, void* meta, void* cuda_stream) {
+int kvb_quantize_chunk_ex(kvb_ctx* c, const void* x, int is_value, int bits, int unrotate_from, int meta_fp16, void* codes,
+                          void* meta, void* cuda_stream) {
   if (!c) return KVB_ERR_INVALID_ARG;
-  if (!x || !codes || !meta || (bits != 4 && bits != 8)) return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");
+  if (!x || !codes || !meta || (bits != 4 && bits != 8) || (meta_fp16 != 0 && meta_fp16 != 1))
+    return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");
+  if (unrotate_from >= 0 && is_value) return fail(c, KVB_ERR_INVALID_ARG, "values are never rotated");
+  if (unrotate_from >= (1 << 24)) return fail(c, KVB_ERR_INVALID_ARG, "position %d out of range [0, 2^24)", unrotate_from);
   if (!aligned16(x) || !aligned16(codes) || !aligned16(meta)) return fail(c, KVB_ERR_BAD_TABLE, "quantize buffers must be 16-byte aligned");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   KVB_CUDA(c, cudaSetDevice(c->device));
   c->last_stream = st;
-  KVB_CUDA(c, launch_quantize(x, is_value ? 1 : 0, bits, codes, meta, c->dims, 0, 0, nullptr, st));
+  KVB_CUDA(c, launch_quantize(x, is_value ? 1 : 0, bits, codes, meta, c->dims, unrotate_from >= 0, unrotate_from >= 0 ? unrotate_from : 0,
+                              c->inv_freq, meta_fp16, st));
   c->launches += 1;
   return KVB_OK;
 }
 
+int kvb_quantize_chunk(kvb_ctx* c, const void* x, int is_value, int bits, void* codes, void* meta, void* cuda_stream) {
+  return kvb_quantize_chunk_ex(c, x, is_value, bits, -1, 0, codes, meta, cuda_stream);
+}
+
 int kvb_quantize_keys_at(kvb_ctx* c, const void* x, int orig_pos, int bits, void* codes, void* meta, void* cuda_stream) {
-  if (!c) return KVB_ERR_INVALID_ARG;
-  if (!x || !codes || !meta || (bits != 4 && bits != 8)) return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");
-  if (orig_pos < 0 || orig_pos >= (1 << 24)) return fail(c, KVB_ERR_INVALID_ARG, "orig_pos=%d out of range [0, 2^24)", orig_pos);
-  if (!aligned16(x) || !aligned16(codes) || !aligned16(meta)) return fail(c, KVB_ERR_BAD_TABLE, "quantize buffers must be 16-byte aligned");
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  KVB_CUDA(c, cudaSetDevice(c->device));
-  c->last_stream = st;
-  KVB_CUDA(c, launch_quantize(x, 0, bits, codes, meta, c->dims, 1, orig_pos, c->inv_freq, st));
-  c->launches += 1;
-  return KVB_OK;
+  if (c && orig_pos < 0) return fail(c, KVB_ERR_INVALID_ARG, "orig_pos=%d out of range [0, 2^24)", orig_pos);
+  return kvb_quantize_chunk_ex(c, x, 0, bits, orig_pos, 0, codes, meta, cuda_stream);
 }
 
 }  // extern "C"

@@ -28,7 +28,7 @@ struct ChunkDesc {
   int32_t delta_pos;     // new_pos - orig_pos
   int32_t mode;
   int32_t tok_offset;    // first token of the request in the call's flat token space
-  int32_t reserved;
+  int32_t meta16;        // (scale, min) pairs are binary16 instead of float32
 };
 
 // One request, as the deviation / top-k / attention kernels see it.
@@ -97,6 +97,6 @@ cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, 
 
 // unrotate != 0 (keys only): rotate by R^(-orig_pos) before quantising (inv_freq: [d/2] doubles, device)
 cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
-                            int unrotate, int orig_pos, const double* inv_freq, cudaStream_t st);
+                            int unrotate, int orig_pos, const double* inv_freq, int meta16, cudaStream_t st);
 
 }  // namespace kvb

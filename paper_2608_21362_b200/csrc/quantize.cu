@@ -24,6 +24,22 @@ __device__ __forceinline__ uint32_t code_of(float v, float mn, float s, float le
   return (uint32_t)c;
 }
 
+// (scale, min) of a group from its extremes.  Compact metadata: min is rounded down to binary16
+// first, the scale is taken against the rounded min and rounded up, so no value leaves the code range.
+__device__ __forceinline__ void group_params(float& mn, float mx, float levels, int meta16, float& s) {
+  if (meta16) mn = __half2float(__float2half_rd(mn));
+  s = mx > mn ? __fdiv_rn(__fsub_rn(mx, mn), levels) : 1.0f;
+  if (meta16) s = __half2float(__float2half_ru(s));
+}
+__device__ __forceinline__ void store_meta(float* meta, size_t pair, float s, float mn, int meta16) {
+  if (meta16) {
+    reinterpret_cast<__half2*>(meta)[pair] = __floats2half2_rn(s, mn);  // both already binary16 values
+  } else {
+    meta[pair * 2 + 0] = s;
+    meta[pair * 2 + 1] = mn;
+  }
+}
+
 // keys: thread = channel (h, j); loops over the tokens of each group.
 // ROT: the chunk was encoded at positions orig_pos..; every key is first rotated back by
 // R_theta^(-orig_pos) (Rotary Positional Embeddings, Eq. 3), so that the stored chunk is position-free
@@ -31,13 +47,14 @@ __device__ __forceinline__ uint32_t code_of(float v, float mn, float s, float le
 // angle, the rotation itself is float32 in a fixed order: u = fma(x, c, +-(x_partner * s)).
 template <int DT, bool ROT>
 __global__ void quantize_k_kernel(const uint16_t* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ meta,
-                                  int C, int E, int bits, int group_tokens, int orig_pos, const double* __restrict__ inv_freq) {
+                                  int C, int E, int bits, int group_tokens, int orig_pos, const double* __restrict__ inv_freq,
+                                  int meta16) {
   const int l = blockIdx.x;
   const int G = C / group_tokens;
   const float levels = (float)((1 << bits) - 1);
   const uint16_t* xl = x + (size_t)l * C * E;
   uint8_t* cl = codes + (size_t)l * C * E * bits / 8;
-  float* ml = meta + (size_t)l * G * E * 2;
+  const size_t pair0 = (size_t)l * G * E;  // first (scale, min) pair of this layer
   for (int c = threadIdx.x; c < E; c += blockDim.x) {  // blockDim.x is even and E is even: c keeps its parity
     float cs = 1.f, sn = 0.f;
     int partner = c;
@@ -61,9 +78,9 @@ __global__ void quantize_k_kernel(const uint16_t* __restrict__ x, uint8_t* __res
         mn = fminf(mn, v);
         mx = fmaxf(mx, v);
       }
-      const float s = mx > mn ? __fdiv_rn(__fsub_rn(mx, mn), levels) : 1.0f;
-      ml[((size_t)g * E + c) * 2 + 0] = s;
-      ml[((size_t)g * E + c) * 2 + 1] = mn;
+      float s;
+      group_params(mn, mx, levels, meta16, s);
+      store_meta(meta, pair0 + (size_t)g * E + c, s, mn, meta16);
       for (int t = g * group_tokens; t < (g + 1) * group_tokens; ++t) {
         const uint32_t q = code_of(value(t), mn, s, levels);
         if (bits == 8) {
@@ -80,7 +97,7 @@ __global__ void quantize_k_kernel(const uint16_t* __restrict__ x, uint8_t* __res
 // values: one warp per (token, head) row of 128 channels, 4 channels per lane
 template <int DT>
 __global__ void quantize_v_kernel(const uint16_t* __restrict__ x, uint8_t* __restrict__ codes, float* __restrict__ meta,
-                                  int C, int H, int bits, int group_ch) {
+                                  int C, int H, int bits, int group_ch, int meta16) {
   const int l = blockIdx.x;
   const int d = 128;
   const int G = d / group_ch;
@@ -101,13 +118,10 @@ __global__ void quantize_v_kernel(const uint16_t* __restrict__ x, uint8_t* __res
       mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
       mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     }
-    const float s = mx > mn ? __fdiv_rn(__fsub_rn(mx, mn), levels) : 1.0f;
+    float s;
+    group_params(mn, mx, levels, meta16, s);
     const int g = (4 * lane) / group_ch;
-    if ((lane % lanes_per_group) == 0) {
-      float* mp = meta + (((size_t)l * C * H + u) * G + g) * 2;
-      mp[0] = s;
-      mp[1] = mn;
-    }
+    if ((lane % lanes_per_group) == 0) store_meta(meta, ((size_t)l * C * H + u) * G + g, s, mn, meta16);
     uint32_t q[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) q[i] = code_of(v[i], mn, s, levels);
@@ -123,30 +137,31 @@ __global__ void quantize_v_kernel(const uint16_t* __restrict__ x, uint8_t* __res
 }  // namespace
 
 cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
-                            int unrotate, int orig_pos, const double* inv_freq, cudaStream_t st) {
+                            int unrotate, int orig_pos, const double* inv_freq, int meta16, cudaStream_t st) {
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   uint8_t* cp = static_cast<uint8_t*>(codes);
   float* mp = static_cast<float*>(meta);
   const int E = m.Hkv * m.d;
+  const bool bf = m.dtype == KVB_DT_BF16;
   if (!is_value) {
     const int gt = bits == 8 ? m.C : m.int4_group;
     if (unrotate) {
-      if (m.dtype == KVB_DT_BF16)
-        quantize_k_kernel<KVB_DT_BF16, true><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, orig_pos, inv_freq);
+      if (bf)
+        quantize_k_kernel<KVB_DT_BF16, true><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, orig_pos, inv_freq, meta16);
       else
-        quantize_k_kernel<KVB_DT_F16, true><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, orig_pos, inv_freq);
+        quantize_k_kernel<KVB_DT_F16, true><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, orig_pos, inv_freq, meta16);
     } else {
-      if (m.dtype == KVB_DT_BF16)
-        quantize_k_kernel<KVB_DT_BF16, false><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, 0, nullptr);
+      if (bf)
+        quantize_k_kernel<KVB_DT_BF16, false><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, 0, nullptr, meta16);
       else
-        quantize_k_kernel<KVB_DT_F16, false><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, 0, nullptr);
+        quantize_k_kernel<KVB_DT_F16, false><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, E, bits, gt, 0, nullptr, meta16);
     }
   } else {
     const int gc = bits == 8 ? m.d : m.int4_group;
-    if (m.dtype == KVB_DT_BF16)
-      quantize_v_kernel<KVB_DT_BF16><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, m.Hkv, bits, gc);
+    if (bf)
+      quantize_v_kernel<KVB_DT_BF16><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, m.Hkv, bits, gc, meta16);
     else
-      quantize_v_kernel<KVB_DT_F16><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, m.Hkv, bits, gc);
+      quantize_v_kernel<KVB_DT_F16><<<m.L, 256, 0, st>>>(xp, cp, mp, m.C, m.Hkv, bits, gc, meta16);
   }
   return cudaGetLastError();
 }

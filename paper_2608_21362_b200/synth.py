@@ -150,6 +150,7 @@ class Chunk:
     v_codes: Optional[torch.Tensor] = None
     k_meta: Optional[torch.Tensor] = None  # f32 [L,G_k,H,d,2]
     v_meta: Optional[torch.Tensor] = None  # f32 [L,C,H,G_v,2]
+    meta_fp16: int = 0  # 1: the two metadata tensors hold binary16 pairs (torch.float16) instead
 
 
 @dataclasses.dataclass
@@ -231,19 +232,21 @@ def materialize(
 # ----------------------------------------------------------------------------------------
 
 
-def assemble_bytes(sh: Shape, plan: RequestPlan) -> int:
-    """Bytes the stitching step must move: packed codes + metadata read, buffer rows written."""
+def assemble_bytes(sh: Shape, plan: RequestPlan, pair_bytes: int = 8) -> int:
+    """Bytes the stitching step must move: packed codes + metadata read, buffer rows written.
+    pair_bytes: size of one (scale, min) pair -- 8 (float32) or 4 (compact binary16 metadata)."""
     E = sh.Hkv * sh.d
+    pb = pair_bytes
     total = 0
     for cp in plan.chunks:
         out_b = 2 * sh.C * E * 2  # K and V rows, 16-bit
         if cp.mode in (MODE_FRESH, MODE_FP16):
             in_b = out_b
         elif cp.mode == MODE_INT8:
-            in_b = 2 * sh.C * E + E * 8 + sh.C * sh.Hkv * 8
+            in_b = 2 * sh.C * E + E * pb + sh.C * sh.Hkv * pb
         else:
             g = sh.int4_group
-            in_b = sh.C * E + (sh.C // g) * E * 8 + sh.C * sh.Hkv * (sh.d // g) * 8
+            in_b = sh.C * E + (sh.C // g) * E * pb + sh.C * sh.Hkv * (sh.d // g) * pb
         total += sh.L * (in_b + out_b)
     return total
 
@@ -253,13 +256,13 @@ def deviation_bytes(sh: Shape, plan: RequestPlan, which: int) -> int:
     return sh.L * nw * plan.T * sh.Hkv * sh.d * 2 * 2  # stored + fresh rows, 16-bit
 
 
-def one_pass_bytes(sh: Shape, plan: RequestPlan, which: int) -> int:
+def one_pass_bytes(sh: Shape, plan: RequestPlan, which: int, pair_bytes: int = 8) -> int:
     """Bytes of the stitch with the deviation sums taken in the same pass: the stitch's own traffic
     plus one read of the fresh rows of every cached chunk (the stored rows are never read back, a
     FRESH chunk's rows are a copy and deviate by nothing)."""
     nw = (which & 1) + ((which >> 1) & 1)
     cached = sum(1 for cp in plan.chunks if cp.mode != MODE_FRESH)
-    return assemble_bytes(sh, plan) + sh.L * nw * cached * sh.C * sh.Hkv * sh.d * 2
+    return assemble_bytes(sh, plan, pair_bytes) + sh.L * nw * cached * sh.C * sh.Hkv * sh.d * 2
 
 
 def attention_flops(sh: Shape, sel) -> int:

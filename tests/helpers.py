@@ -46,6 +46,8 @@ def oracle_chunk_dicts(chunks):
             t = getattr(ck, name)
             if t is None:
                 d[name] = None
+            elif name.endswith("_meta"):  # compact (binary16) pairs reach the oracle as the float32 values they hold
+                d[name] = t.detach().cpu().float().numpy()
             elif t.dtype in (torch.bfloat16, torch.float16):
                 d[name] = bits_of(t)
             else:

@@ -490,3 +490,40 @@ def test_unrotate_keys_is_the_inverse_rotation_in_float32():
     u = oracle.unrotate_keys(oracle.round_to_bits(e, 1), 1, theta, 1000)[0, 0]
     assert u[0] == np.float32(math.cos(1000.0)) and u[d // 2] == -np.float32(math.sin(1000.0))
     assert np.all(u[1 : d // 2] == 0) and np.all(u[d // 2 + 1 :] == 0)
+
+
+# ------------------------------------------------------------------ Eq. 6 with compact (binary16) metadata
+def test_compact_metadata_quantiser_rounds_outward_and_keeps_the_error_bound():
+    r = np.random.default_rng(77)
+    x = oracle.bits_to_f64(oracle.round_to_bits(r.standard_normal((64, 2, 32)) * np.exp(r.uniform(-3, 3, (1, 2, 32))), 1), 1)
+    for bits, levels in ((8, 255), (4, 15)):
+        for which in ("k", "v"):
+            if which == "k":
+                codes, meta = oracle.quantize_k(x, bits, 32, meta16=True)
+                c0, m0 = oracle.quantize_k(x, bits, 32)
+                deq = oracle.dequant_k(codes, meta, 32, bits, 32)
+                grp_min = x.reshape(2, 32, 2, 32).min(axis=1)        # [G,H,d]
+                grp_max = x.reshape(2, 32, 2, 32).max(axis=1)
+                s_of = np.repeat(meta[..., 0], 32, axis=0).astype(np.float64)
+            else:
+                codes, meta = oracle.quantize_v(x, bits, 16, meta16=True)
+                c0, m0 = oracle.quantize_v(x, bits, 16)
+                deq = oracle.dequant_v(codes, meta, 32, bits, 16)
+                grp_min = x.reshape(64, 2, 2, 16).min(axis=3)        # [C,H,G]
+                grp_max = x.reshape(64, 2, 2, 16).max(axis=3)
+                s_of = np.repeat(meta[..., 0], 16, axis=2).astype(np.float64)
+            s16, m16 = meta[..., 0], meta[..., 1]
+            # the stored pair is binary16; min is the largest binary16 value not above the true minimum
+            assert np.array_equal(meta, meta.astype(np.float16).astype(np.float32))
+            assert np.all(m16 <= grp_min)
+            above = np.nextafter(m16.astype(np.float16), np.float16(np.inf)).astype(np.float64)
+            assert np.all(above > grp_min)
+            # scale is the smallest binary16 value not below (max - min16)/levels (float32 division)
+            want = ((grp_max.astype(np.float32) - m16) / np.float32(levels)).astype(np.float32)
+            assert np.all(s16 >= want)
+            below = np.nextafter(s16.astype(np.float16), np.float16(-np.inf)).astype(np.float32)
+            assert np.all(below < want)
+            # so every value is inside the code range and the error stays half a (rounded) step
+            assert np.all(np.abs(deq - x) <= 0.5 * s_of * (1 + 1e-6) + 1e-12)
+            # and the float32 variant is untouched by the option
+            assert np.array_equal(c0, (oracle.quantize_k(x, bits, 32) if which == "k" else oracle.quantize_v(x, bits, 16))[0])
