@@ -2,7 +2,8 @@
 """Benchmark of the KV-chunk stitching path on B200.
 
 A step is one pass of the whole path over one batch of synthetic requests:
-    kvb_assemble -> kvb_deviation_topk -> kvb_selective_attn
+    kvb_assemble_select (stitch + deviation sums in one kernel, then the selection) -> kvb_selective_attn
+(`--path two-call`: kvb_assemble -> kvb_deviation_topk -> kvb_selective_attn, the same work in three calls)
 Default workload (N=1): the Qwen2.5-3B-shaped 2048-token prompt (12 int8 chunks + 4 fresh), one
 request per step, rotating through enough independent replicas that the working set is far
 larger than L2.  `--workload cfg2|cfg4` selects the long int4 prompt (with its selective
@@ -449,7 +450,8 @@ def main():
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed ncu captures
     # (profiles/cfg1_launches_and_kernels.md, profiles/cfg2_kernels.md); null where none was taken
     ncu_traffic = {
-        ("cfg1_qwen3b_2k_int8", "selective_attn"): 207.0e6, ("cfg1_qwen3b_2k_int8", "assemble"): 67.6e6,
+        ("cfg1_qwen3b_2k_int8", "selective_attn"): 208.2e6, ("cfg1_qwen3b_2k_int8", "assemble"): 67.6e6,
+        ("cfg1_qwen3b_2k_int8", "assemble_select"): 126.6e6,
         ("cfg1_qwen3b_2k_int8", "deviation_topk"): 154.2e6, ("cfg2_long_int4_8k", "selective_attn"): 647.1e6,
         ("cfg2_long_int4_8k", "assemble"): 381.0e6, ("cfg2_long_int4_8k", "deviation_topk"): 608.2e6,
     }
