@@ -258,7 +258,12 @@ int kvb_validate(const kvb_model_desc* model, const kvb_limits* limits, const kv
 /* floor(ratio * T), the k of Algorithm 2 step 3. */
 int kvb_select_count(int T, double ratio);
 
-/* Synchronises the context's last stream and returns the sticky device status (0 = clean). */
+/* Synchronises the context's last stream and reports the device status word:
+ * KVB_OK if no kernel flagged anything since the last report, else
+ * KVB_ERR_DEVICE_STATUS with the bits in kvb_last_error's text (0x1 a bounded
+ * wait ran out, 0x2 a descriptor failed a device-side check, 0x4 a selection
+ * did not fit sel_capacity and was cut to its first sel_capacity entries).
+ * Reporting clears the word, so the context stays usable. */
 int kvb_last_status(kvb_ctx* ctx);
 /* Text of the last host-side error of this context (valid until the next call). */
 const char* kvb_last_error(kvb_ctx* ctx);

@@ -37,7 +37,6 @@ constexpr uint32_t kSubBytes = kSubKeys * kD * 2;    // 16 KB: one stream's K or
 constexpr uint32_t kTmemCols = 256;                  // S/P: columns 0..127, O: columns 128..255
 constexpr uint32_t kWaitLimit = 1u << 24;
 constexpr float kLazyThreshold = 8.0f;
-constexpr bool kPolyExp = false;  // one exp2 in four goes to the FMA pipe
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -146,13 +145,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
       "r"(r[31])
       : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]),
-      "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptors (128-byte swizzle, 8-row groups 1024 bytes apart).
@@ -184,20 +176,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
-}
-
-// 2^x on the FMA and integer pipes (no MUFU): round to the nearest integer with the 1.5*2^23 trick,
-// a cubic for 2^f on [-0.5, 0.5] (relative error 7.5e-5, far below the 16-bit rounding of P), and
-// the integer part added into the exponent field.  Used for a fraction of the scores so that the
-// 16-per-clock special-function unit is not the limiter.
-__device__ __forceinline__ float poly_exp2(float x) {
-  x = fmaxf(x, -125.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.05517165f, f, 0.24261113f);
-  p = fmaf(p, f, 0.69326097f);
-  p = fmaf(p, f, 0.99992806f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
 
 // Packed float32 pairs (one instruction for two lanes of work) and the three-input maximum.
@@ -600,7 +578,7 @@ __global__ void __launch_bounds__(kThreads, 2)
         f2_unpack(f2_fma(f2_pack(__uint_as_float(r0[i]), __uint_as_float(r0[i + 1])), scale2, negm2), a0, a1);
         f2_unpack(f2_fma(f2_pack(__uint_as_float(r1[i]), __uint_as_float(r1[i + 1])), scale2, negm2), a2, a3);
         const float p0 = fast_exp2(a0), p1 = fast_exp2(a1), p2 = fast_exp2(a2);
-        const float p3 = kPolyExp ? poly_exp2(a3) : fast_exp2(a3);
+        const float p3 = fast_exp2(a3);
         ps2[(i >> 1) & 1] = f2_add(ps2[(i >> 1) & 1], f2_pack(p0, p1));
         ps2[2 + ((i >> 1) & 1)] = f2_add(ps2[2 + ((i >> 1) & 1)], f2_pack(p2, p3));
         pk[i >> 1] = pack2<DT>(p0, p1);

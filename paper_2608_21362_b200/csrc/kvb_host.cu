@@ -260,7 +260,12 @@ int kvb_last_status(kvb_ctx* c) {
   KVB_CUDA(c, cudaStreamSynchronize(c->last_stream));
   uint32_t st = 0;
   KVB_CUDA(c, cudaMemcpy(&st, c->status_dev, sizeof(st), cudaMemcpyDeviceToHost));
-  if (st) return fail(c, KVB_ERR_DEVICE_STATUS, "device status word 0x%x", st);
+  if (st) {
+    KVB_CUDA(c, cudaMemset(c->status_dev, 0, sizeof(st)));  // reported once; the context stays usable
+    return fail(c, KVB_ERR_DEVICE_STATUS, "device status word 0x%x%s%s%s", st, (st & DEV_STATUS_WAIT_TIMEOUT) ? " (a bounded wait ran out)" : "",
+                (st & DEV_STATUS_BAD_DESC) ? " (a descriptor failed a device-side check)" : "",
+                (st & DEV_STATUS_SEL_OVERFLOW) ? " (a selection did not fit sel_capacity)" : "");
+  }
   return KVB_OK;
 }
 

@@ -122,6 +122,38 @@ def test_attention_sink_tokens_join_the_selection():
         B.kvb_destroy(ctx)
 
 
+def test_selection_overflow_is_reported_once_and_cut_cleanly():
+    """sel_capacity = k passes the host check, but the seam windows add positions: the kernel keeps
+    the first sel_capacity entries of the ascending union, sets the status word, and the next
+    report is clean again (no trap, the context stays usable)."""
+    wl = synth.workload(0)
+    sh = wl.shape
+    reqs = prepare(wl)
+    (r,) = reqs
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        k = B.kvb_select_count(r.plan.T, 0.15)
+        sel = B.SelectionTable([r.plan.T], [k], [k], DEV)  # room for the top-k only
+        guard = torch.full((k + 64,), -7, dtype=torch.int32, device=DEV)
+        sel.sel[0] = guard[:k]
+        sel.array[0].sel = guard.data_ptr()
+        B.kvb_deviation_topk(ctx, tbl, 0.15, -1, 16, 0, 3, sel)
+        assert B.kvb_last_status(ctx, check=False) == B.KVB_ERR_DEVICE_STATUS
+        assert "0x4" in B.kvb_last_error(ctx) and "sel_capacity" in B.kvb_last_error(ctx)
+        assert int(sel.n_sel[0]) == k
+        rank = sel.rank[0].cpu().numpy()[:k]
+        want = oracle.seam_select(rank, [c.plan.new_pos for c in r.chunks], [c.plan.mode for c in r.chunks], r.plan.T, 16, 0)
+        assert len(want) > k
+        assert np.array_equal(guard[:k].cpu().numpy(), want[:k])
+        assert torch.all(guard[k:] == -7), "nothing may be written past sel_capacity"
+        assert B.kvb_last_status(ctx, check=False) == B.KVB_OK  # reported once
+        sel2, ks, caps = run_select(ctx, wl, reqs, tbl, use_oracle_buffer=False)  # a correct call afterwards
+        check_selection(sh, reqs, sel2, ks, wl.select)
+    finally:
+        B.kvb_destroy(ctx)
+
+
 def test_attention_persistent_and_one_tile_ctas_agree(monkeypatch):
     """The attention kernel runs either as persistent CTAs drawing tiles from a counter (short prompts)
     or with one tile per CTA (long prompts); KVB_ATTN forces either.  Both must give the same bits, on
