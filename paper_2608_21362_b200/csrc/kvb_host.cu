@@ -38,6 +38,7 @@ struct kvb_ctx {
   int n_sm = 0;
   bool attn_legacy = false;  // KVB_ATTN=mma selects the warp-level mma.sync kernel (debug aid)
   int attn_mode = 0;         // KVB_ATTN=onetile (2): one tile per CTA instead of persistent CTAs (cross-check)
+  bool force_copy = false;   // KVB_DESC=copy: descriptors always go by cudaMemcpyAsync (cross-check)
   cudaStream_t last_stream = nullptr;
   int64_t launches = 0;
   char err[512] = {0};
@@ -76,7 +77,19 @@ int take_slot(kvb_ctx* c, uint8_t** host) {
   return -(s + 1);  // negative = success, encodes the slot
 }
 
-int upload(kvb_ctx* c, int slot, const uint8_t* host, size_t bytes, cudaStream_t st) {
+// Sends the call's packed tables to the device arena.  Small tables ride in a kernel argument (the
+// launch reads the host bytes before it returns, so the staging slot is free again at once) and, when
+// rope_chunks > 0, the same kernel fills the rotation table: *rope_done tells the caller.  Larger
+// tables are copied from the pinned slot, guarded by the slot's event.
+int upload(kvb_ctx* c, int slot, const uint8_t* host, size_t bytes, cudaStream_t st, int rope_chunks = 0, bool* rope_done = nullptr) {
+  if (rope_done) *rope_done = false;
+  if (bytes <= kDescBlobBytes && !c->force_copy) {
+    KVB_CUDA(c, launch_store_blob(host, bytes, c->arena_dev, rope_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+    c->slot_used[slot] = false;
+    c->launches += 1;
+    if (rope_done) *rope_done = rope_chunks > 0;
+    return KVB_OK;
+  }
   KVB_CUDA(c, cudaMemcpyAsync(c->arena_dev, host, bytes, cudaMemcpyHostToDevice, st));
   KVB_CUDA(c, cudaEventRecord(c->slot_done[slot], st));
   c->slot_used[slot] = true;
@@ -215,6 +228,8 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, attention_tc_configure());
   const char* attn_env = getenv("KVB_ATTN");
   c->attn_legacy = attn_env && strcmp(attn_env, "mma") == 0;
+  const char* desc_env = getenv("KVB_DESC");
+  c->force_copy = desc_env && strcmp(desc_env, "copy") == 0;
   c->attn_mode = attn_env && strcmp(attn_env, "persistent") == 0 ? 1 : (attn_env && strcmp(attn_env, "onetile") == 0 ? 2 : 0);
 
   const int half = m.d / 2;
@@ -396,13 +411,17 @@ int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stre
   if (slot_code >= 0) return slot_code;
   const int slot = -slot_code - 1;
   const size_t smem = pack_chunks(c, reqs, n_req, reinterpret_cast<ChunkDesc*>(host));
-  const int up = upload(c, slot, host, sizeof(ChunkDesc) * (size_t)n_chunks, st);
+  bool rope_done = false;
+  const int up = upload(c, slot, host, sizeof(ChunkDesc) * (size_t)n_chunks, st, n_chunks, &rope_done);
   if (up != KVB_OK) return up;
   c->last_stream = st;
   const ChunkDesc* cd_dev = reinterpret_cast<const ChunkDesc*>(c->arena_dev);
-  KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+  if (!rope_done) {
+    KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+    c->launches += 1;
+  }
   KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, 0, nullptr, st));
-  c->launches += 2;
+  c->launches += 1;
   return KVB_OK;
 }
 
@@ -469,19 +488,23 @@ int kvb_assemble_select(kvb_ctx* c, const kvb_request* reqs, int n_req, const kv
   if (st2 != KVB_OK) return st2;
   const int st3 = clear_acc_if_dirty(c, st);
   if (st3 != KVB_OK) return st3;
-  const int up = upload(c, slot, host, sw_off + sizeof(SeamWindow) * (size_t)ext.n_seams, st);
+  bool rope_done = false;
+  const int up = upload(c, slot, host, sw_off + sizeof(SeamWindow) * (size_t)ext.n_seams, st, n_chunks, &rope_done);
   if (up != KVB_OK) return up;
   c->last_stream = st;
   const ChunkDesc* cd_dev = reinterpret_cast<const ChunkDesc*>(c->arena_dev);
   const ReqDesc* rd_dev = reinterpret_cast<const ReqDesc*>(c->arena_dev + rd_off);
   const SeamWindow* sw_dev = reinterpret_cast<const SeamWindow*>(c->arena_dev + sw_off);
-  KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+  if (!rope_done) {
+    KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+    c->launches += 1;
+  }
   c->acc_dirty = true;  // cleared again once both kernels are in the stream
   KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, p->which, c->acc, st));
   KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_deviation_terms(c, p->which), ext.max_T, ext.max_k, c->acc,
                           c->status_dev, st));
   c->acc_dirty = false;
-  c->launches += 3;
+  c->launches += 2;
   return KVB_OK;
 }
 

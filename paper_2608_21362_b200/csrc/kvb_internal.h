@@ -60,6 +60,12 @@ struct ModelDims {
 };
 
 // ---- launchers (each defined next to its kernel) ----
+// Tables of at most kDescBlobBytes go to the arena as a kernel argument (csrc/desc_store.cu); the
+// chunk descriptors, if any, must be at the start of the bytes, and n_rope_chunks > 0 also fills
+// cs_table[n_rope_chunks][half_d] from their delta_pos.
+constexpr size_t kDescBlobBytes = 3840;
+cudaError_t launch_store_blob(const void* host_bytes, size_t bytes, uint8_t* dst, int n_rope_chunks, const double* inv_freq,
+                              int half_d, float2* cs_table, cudaStream_t st);
 // launch_assemble: acc != NULL fuses the deviation sums (which: bit 0 keys, bit 1 values) into the stitch.
 cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const double* inv_freq, int half_d,
                               float2* cs_table, cudaStream_t st);

@@ -122,6 +122,38 @@ def test_attention_sink_tokens_join_the_selection():
         B.kvb_destroy(ctx)
 
 
+def test_descriptor_upload_paths_agree(monkeypatch):
+    """Small calls send their tables as a kernel argument (and fill the rotation table in the same
+    launch); KVB_DESC=copy forces the pinned-buffer copy and the separate table kernel.  Same bits."""
+    wl = synth.workload(0)
+    sh = wl.shape
+    got = {}
+    for mode in ("kernel", "copy"):
+        if mode == "copy":
+            monkeypatch.setenv("KVB_DESC", "copy")
+        else:
+            monkeypatch.delenv("KVB_DESC", raising=False)
+        reqs = prepare(wl)
+        (r,) = reqs
+        ctx = B.create_for_shape(sh, 0)
+        try:
+            before = B.kvb_launch_count(ctx)
+            tbl = B.RequestTable(reqs)
+            k = B.kvb_select_count(r.plan.T, 0.15)
+            sel = B.SelectionTable([r.plan.T], [k], [r.sel_capacity], DEV)
+            B.kvb_assemble_select(ctx, tbl, 0.15, -1, 16, 0, 3, sel)
+            out = torch.zeros_like(r.q)
+            B.kvb_selective_attn(ctx, tbl, sel, [r.q], [out], 0.1)
+            B.kvb_last_status(ctx)
+            # kernel path: store+table, stitch, selection; store, attention.  copy path: table, stitch, selection; attention
+            assert B.kvb_launch_count(ctx) - before == (5 if mode == "kernel" else 4)
+            got[mode] = (r.kv_buf.view(torch.int16).clone(), sel.delta[0].clone(), sel.sel[0].clone(), out.view(torch.int16).clone())
+        finally:
+            B.kvb_destroy(ctx)
+    for a, b in zip(got["kernel"], got["copy"]):
+        assert torch.equal(a, b)
+
+
 def test_selection_overflow_is_reported_once_and_cut_cleanly():
     """sel_capacity = k passes the host check, but the seam windows add positions: the kernel keeps
     the first sel_capacity entries of the ascending union, sets the status word, and the next
