@@ -445,6 +445,8 @@ def main():
         }
     for s in stages.values():
         s["frac"] = s["achieved"] / s["peak"]
+        # context only: fraction of the nominal figure (8 TB/s HBM3e, 2250 TFLOP/s dense bf16)
+        s["frac_of_nominal"] = s["achieved"] / (8000.0 if s["bound"] == "hbm" else 2250.0)
     top = max(stages, key=lambda k: stages[k]["ms"])
     roof = {k: stages[top][k] for k in ("bound", "achieved", "peak", "unit", "frac")}
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed ncu captures
