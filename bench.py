@@ -496,6 +496,13 @@ def main():
             "value": tok_s / (secs * sh.L / n_l), "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": "%d request(s), %d tokens, %d of %d layers, all stages and all selected rows; %.1f s measured, scaled by layers" % (len(reqs_host), tok_s, n_l, sh.L, secs),
         }
+        if t1 * threads <= 12.0:  # one core as well, where a single layer stays within a few seconds
+            import oracle
+
+            oracle.set_threads(1)
+            s1 = oracle_sample_seconds(wl, reqs_host, 1)[0]
+            oracle.set_threads(threads)
+            line["cpu_baseline"]["value_1_core"] = tok_s / (s1 * sh.L)
     B.kvb_destroy(ctx)
     if rank == 0:
         print(json.dumps(line))

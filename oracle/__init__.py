@@ -80,6 +80,11 @@ def max_threads() -> int:
     return int(lib().kvo_max_threads())
 
 
+def set_threads(n: int) -> None:
+    """Threads the oracle's parallel loops use from now on (for one-core vs all-core timings)."""
+    lib().kvo_set_threads(int(n))
+
+
 # ---------------------------------------------------------------- 16-bit formats
 def round_to_bits(x, dtype: int) -> np.ndarray:
     """float64 array -> uint16 bit patterns of bf16 / fp16 (nearest-even, one rounding)."""

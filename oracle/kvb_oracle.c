@@ -563,6 +563,16 @@ int kvo_max_threads(void) {
 #endif
 }
 
+/* Number of threads the parallel loops may use from now on (timing on one core vs all cores). */
+void kvo_set_threads(int n) {
+#ifdef _OPENMP
+  extern void omp_set_num_threads(int);
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
 /* ------------------------------------------------------------------ */
 /* Algorithm 2, step 4 (and Algorithm 1's splice): patch                */
 /* ------------------------------------------------------------------ */
