@@ -74,6 +74,8 @@ __global__ void __launch_bounds__(kThreads, 1)
   uint32_t* s_mask = s_keys + t_pad;                                                      // [kThreads] selection bitmask
   unsigned long long* s_comp = reinterpret_cast<unsigned long long*>(s_mask + kThreads);  // [k_pad]
   __shared__ uint32_t s_warp_sums[33];
+  __shared__ uint32_t s_eqm[kThreads];   // per word of 32 positions: keys equal to the threshold
+  __shared__ uint32_t s_base[kThreads];  // per word: how many selected positions precede it
   __shared__ uint32_t s_hist[2][256];  // two buffers: one is cleared while the other is scanned
   __shared__ uint32_t s_pick[2];       // chosen bin, remaining need
 
@@ -149,26 +151,24 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
   }
 
-  // ---- 3. the top-k set in index order; thread w owns positions 32w .. 32w+31 (read in a
-  //      lane-rotated order so that the 32 lanes of a warp hit 32 different banks)
-  uint32_t gt_mask = 0, eq_mask = 0;
-  {
-    const int base = tid * 32;
-    if (k >= T) {
-      for (int i = 0; i < 32; ++i)
-        if (base + i < T) gt_mask |= 1u << i;
-    } else if (k > 0 && base < T) {
-#pragma unroll 8
-      for (int j = 0; j < 32; ++j) {
-        const int i = (j + lane) & 31;
-        if (base + i < T) {
-          const uint32_t key = s_keys[base + i];
-          if (key > prefix) gt_mask |= 1u << i;
-          if (key == prefix) eq_mask |= 1u << i;
-        }
-      }
+  // ---- 3. the top-k set in index order.  Positions go by words of 32: a warp votes a word's
+  //      "above the threshold" and "equal to it" masks, thread w then owns word w for the prefix
+  //      scan, and warps write the word's selected positions side by side.
+  const int n_words = (T + 31) >> 5;  // <= kThreads
+  const uint32_t lanes_below = (1u << lane) - 1u;
+  for (int w = warp; w < n_words; w += kThreads / 32) {
+    const int t = w * 32 + lane;
+    const bool live = t < T;
+    const uint32_t key = live ? s_keys[t] : 0u;
+    const uint32_t gt = __ballot_sync(0xffffffffu, live && (k >= T || (k > 0 && key > prefix)));
+    const uint32_t eq = __ballot_sync(0xffffffffu, live && k > 0 && k < T && key == prefix);
+    if (lane == 0) {
+      s_mask[w] = gt;
+      s_eqm[w] = eq;
     }
   }
+  __syncthreads();
+  const uint32_t gt_mask = tid < n_words ? s_mask[tid] : 0u, eq_mask = tid < n_words ? s_eqm[tid] : 0u;
   // one scan for both counts (each at most 32768: 16 bits apiece)
   uint32_t tot_packed;
   const uint32_t packed_before =
@@ -177,34 +177,67 @@ __global__ void __launch_bounds__(kThreads, 1)
   const uint32_t n_take_eq = (k > 0 && k < T) ? need : 0u;  // threshold-valued keys taken, lowest indices first
   int k_pad = 1;
   while (k_pad < k) k_pad <<= 1;
-  // composite sort keys (larger delta first, then lower index) of the selected positions, in index order
-  {
-    uint32_t sel_mask = gt_mask;
-    uint32_t e = eq_mask, r = eq_before;
-    while (e) {
-      const int b = __ffs(e) - 1;
-      e &= e - 1;
-      if (r < n_take_eq) sel_mask |= 1u << b;
-      ++r;
-    }
-    uint32_t pos = gt_before + min(eq_before, n_take_eq);
-    uint32_t m2 = sel_mask;
-    while (m2) {
-      const int b = __ffs(m2) - 1;
-      m2 &= m2 - 1;
-      const uint32_t t = tid * 32 + b;
-      if (pos < (uint32_t)k_pad) s_comp[pos] = ((unsigned long long)(~s_keys[t]) << 32) | t;
-      ++pos;
+  if (tid < n_words) {
+    // of this word's threshold-valued positions the lowest `take` join the selection
+    uint32_t sel_mask = gt_mask, e = eq_mask;
+    int take = (int)min((uint32_t)__popc(eq_mask), n_take_eq > eq_before ? n_take_eq - eq_before : 0u);
+    while (take-- > 0) {
+      const uint32_t low = e & (0u - e);
+      sel_mask |= low;
+      e ^= low;
     }
     s_mask[tid] = sel_mask;
+    s_base[tid] = gt_before + min(eq_before, n_take_eq);
   }
   for (int i = k + tid; i < k_pad; i += kThreads) s_comp[i] = ~0ull;  // padding sorts last
   const uint32_t tot_sel = (tot_packed & 0xFFFFu) + min(tot_packed >> 16, n_take_eq);
   __syncthreads();
+  // composite sort keys (larger delta first, then lower index) of the selected positions, in index order
+  for (int w = warp; w < n_words; w += kThreads / 32) {
+    const uint32_t m = s_mask[w];
+    if ((m >> lane) & 1u) {
+      const uint32_t pos = s_base[w] + __popc(m & lanes_below);
+      const uint32_t t = w * 32 + lane;
+      if (pos < (uint32_t)k_pad) s_comp[pos] = ((unsigned long long)(~s_keys[t]) << 32) | t;
+    }
+  }
+  __syncthreads();
 
   // ---- bitonic sort of s_comp[0..k_pad): element i lives in lane i % 32 of its warp for the steps
   //      with stride < 32 (registers + shuffles); larger strides go through shared memory
-  if (k_pad >= 32) {
+  if (k_pad >= 64 && k_pad <= kThreads && (size_t)k_pad * 8 <= (size_t)t_pad * 4) {
+    // One element per thread, held in a register for the whole sort.  Strides below 32 are shuffles;
+    // larger strides publish the element and read the partner's, alternating between s_comp and the
+    // key array (no longer needed) so that one barrier per step is enough.  Only the k_pad threads
+    // that hold an element take part (named barrier 1).
+    if (tid < k_pad) {
+      unsigned long long* bufs[2] = {s_comp, reinterpret_cast<unsigned long long*>(s_keys)};
+      unsigned long long v = s_comp[tid];
+#pragma unroll
+      for (int size = 2; size <= 32; size <<= 1) {
+        const bool up = (tid & size) == 0;
+#pragma unroll
+        for (int stride = size >> 1; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+      }
+      int b = 1;
+      for (int size = 64; size <= k_pad; size <<= 1) {
+        const bool up = (tid & size) == 0;
+        for (int stride = size >> 1; stride >= 32; stride >>= 1) {
+          bufs[b][tid] = v;
+          asm volatile("bar.sync 1, %0;" ::"r"(k_pad) : "memory");
+          const unsigned long long o = bufs[b][tid ^ stride];
+          const bool take_min = ((tid & stride) == 0) == up;
+          v = take_min ? (v < o ? v : o) : (v > o ? v : o);
+          b ^= 1;
+        }
+#pragma unroll
+        for (int stride = 16; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+      }
+      asm volatile("bar.sync 1, %0;" ::"r"(k_pad) : "memory");  // the last partner reads are done
+      s_comp[tid] = v;
+    }
+    __syncthreads();
+  } else if (k_pad >= 32) {
     for (int i0 = 0; i0 < k_pad; i0 += kThreads) {  // sizes 2..32 entirely in registers
       const int i = i0 + tid;
       if (i0 + (tid & ~31) >= k_pad) break;  // whole warps only (k_pad is a multiple of 32)
@@ -259,21 +292,28 @@ __global__ void __launch_bounds__(kThreads, 1)
   for (int i = tid; i < k; i += kThreads) rq.rank[i] = (int32_t)(uint32_t)(s_comp[i] & 0xFFFFFFFFull);
 
   // ---- 4. union with the seam windows, ascending list
-  for (int w = 0; w < rq.n_seams; ++w) {
+  //      (a warp per window, a lane per mask word of the window)
+  for (int w = warp; w < rq.n_seams; w += kThreads / 32) {
     const SeamWindow sw = seams[rq.seam_offset + w];
-    for (int t = sw.lo + tid; t < sw.hi; t += kThreads) atomicOr(&s_mask[t >> 5], 1u << (t & 31));
+    if (sw.hi <= sw.lo) continue;
+    const int last = (sw.hi - 1) >> 5;
+    for (int j = (sw.lo >> 5) + lane; j <= last; j += 32) {
+      const int lo_bit = max(sw.lo - j * 32, 0), hi_bit = min(sw.hi - j * 32, 32);  // bits [lo_bit, hi_bit) of word j
+      const uint32_t upto = hi_bit >= 32 ? 0xFFFFFFFFu : ((1u << hi_bit) - 1u);
+      atomicOr(&s_mask[j], upto & ~((1u << lo_bit) - 1u));
+    }
   }
   __syncthreads();
-  const uint32_t word = s_mask[tid];
+  const uint32_t word = tid < n_words ? s_mask[tid] : 0u;
   uint32_t n_sel;
-  uint32_t pos = block_exclusive_scan(__popc(word), s_warp_sums, &n_sel);
-  {
-    uint32_t e = word;
-    while (e) {
-      const int b = __ffs(e) - 1;
-      e &= e - 1;
-      if (pos < (uint32_t)rq.sel_capacity) rq.sel[pos] = tid * 32 + b;
-      ++pos;
+  const uint32_t word_base = block_exclusive_scan(__popc(word), s_warp_sums, &n_sel);
+  if (tid < n_words) s_base[tid] = word_base;
+  __syncthreads();
+  for (int w = warp; w < n_words; w += kThreads / 32) {
+    const uint32_t m = s_mask[w];
+    if ((m >> lane) & 1u) {
+      const uint32_t pos = s_base[w] + __popc(m & lanes_below);
+      if (pos < (uint32_t)rq.sel_capacity) rq.sel[pos] = w * 32 + lane;
     }
   }
   if (tid == 0) {

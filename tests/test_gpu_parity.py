@@ -387,7 +387,9 @@ def test_ragged_batch_pipeline():
             rows = np.sort(rng.choice(n, size=min(n, 24), replace=False)).astype(np.int32)
             rows[-1] = n - 1
             check_attention(sh, r, sel_idx, outs[i], [0, int(rng.integers(1, sh.L))], rows)
-        assert B.kvb_launch_count(ctx) == 5
+        # the whole batch goes in a fixed number of launches, whatever the number of requests: table +
+        # stitch, (store) + deviation + selection, (store) + attention
+        assert 5 <= B.kvb_launch_count(ctx) <= 7
     finally:
         B.kvb_destroy(ctx)
 
