@@ -17,6 +17,7 @@
 #include "deviation_math.cuh"
 #include "f32x2.cuh"
 #include "kvb_internal.h"
+#include "pdl.cuh"
 
 namespace kvb {
 namespace {
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__(kThreads, 3)
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) uint64_t bars[kParts + 1];
 
+  pdl_wait();  // the descriptors and the rotation table come from the kernel before this one
   const int tid = threadIdx.x;
   const int H = m.Hkv;
   const int split = assemble_split(H);  // CTAs per chunk-layer, so that a CTA stages at most 256 rows
@@ -518,14 +520,14 @@ cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2*
   const bool dev = acc != nullptr && (which & 3);
   if (m.dtype == KVB_DT_BF16) {
     if (dev)
-      assemble_kernel<__nv_bfloat16, true><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, which, acc);
+      return launch_pdl(assemble_kernel<__nv_bfloat16, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
     else
-      assemble_kernel<__nv_bfloat16, false><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, 0, nullptr);
+      return launch_pdl(assemble_kernel<__nv_bfloat16, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
   } else {
     if (dev)
-      assemble_kernel<__half, true><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, which, acc);
+      return launch_pdl(assemble_kernel<__half, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
     else
-      assemble_kernel<__half, false><<<grid, kThreads, smem_bytes, st>>>(chunks, cs_table, m, status, 0, nullptr);
+      return launch_pdl(assemble_kernel<__half, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
   }
   return cudaGetLastError();
 }

@@ -23,6 +23,7 @@
 #include <cuda_fp16.h>
 
 #include "kvb_internal.h"
+#include "pdl.cuh"
 
 namespace kvb {
 namespace {
@@ -313,7 +314,11 @@ __global__ void __launch_bounds__(kThreads, 2)
   // The producer thread looks up its first tile before the CTA-wide sync, under the barrier
   // initialisation and the TMEM allocation (done by other warps).
   unsigned int drawn = 0xFFFFFFFFu;  // only the producer thread draws
-  if (tid == 0) drawn = PERSISTENT ? atomicAdd(tile_counter, 1u) : blockIdx.x;
+  if (tid == 0) {
+    pdl_wait();  // descriptors, tensor maps and the tile counter come from the kernel before this one; the
+                 // other roles touch global memory only after this thread has published a tile
+    drawn = PERSISTENT ? atomicAdd(tile_counter, 1u) : blockIdx.x;
+  }
   auto decode_next = [&]() { return decode_next_tile<PERSISTENT>(drawn, tile_counter, reqs, maps, n_req, total_tiles, per_tile, TOK, m.Hkv); };
   NextTile next;
   next.ti.nsb = 0;
@@ -703,15 +708,15 @@ cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req
   if (persistent) {  // two CTAs per SM; each takes tiles from *tile_counter (zero at launch) until they run out
     const unsigned grid = (unsigned)(work < 2LL * n_sm ? work : 2LL * n_sm);
     if (m.dtype == KVB_DT_BF16)
-      attn_tc_kernel<KVB_DT_BF16, true><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(attn_tc_kernel<KVB_DT_BF16, true>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
     else
-      attn_tc_kernel<KVB_DT_F16, true><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(attn_tc_kernel<KVB_DT_F16, true>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
   } else {
     const unsigned grid = (unsigned)work;
     if (m.dtype == KVB_DT_BF16)
-      attn_tc_kernel<KVB_DT_BF16, false><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(attn_tc_kernel<KVB_DT_BF16, false>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
     else
-      attn_tc_kernel<KVB_DT_F16, false><<<grid, kThreads, kSmemBytes, st>>>(reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(attn_tc_kernel<KVB_DT_F16, false>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
   }
   return cudaGetLastError();
 }

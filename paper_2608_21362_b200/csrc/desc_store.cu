@@ -8,6 +8,7 @@
 #include <string.h>
 
 #include "kvb_internal.h"
+#include "pdl.cuh"
 
 namespace kvb {
 namespace {
@@ -19,6 +20,8 @@ struct DescBlob {
 __global__ void __launch_bounds__(128)
     store_blob_kernel(const __grid_constant__ DescBlob blob, int n16, uint4* __restrict__ dst, int n_chunks,
                       const double* __restrict__ inv_freq, int half_d, float2* __restrict__ cs_table) {
+  pdl_trigger();  // the call's next kernel may set itself up while this one runs
+  pdl_wait();     // the previous call's kernels may still be reading the arena
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n16) dst[i] = blob.v[i];
   if (i < n_chunks * half_d) {  // the chunk descriptors sit at the start of the blob
@@ -40,9 +43,8 @@ cudaError_t launch_store_blob(const void* host_bytes, size_t bytes, uint8_t* dst
   if (padded > bytes) memset(reinterpret_cast<uint8_t*>(&blob) + bytes, 0, padded - bytes);
   const int n16 = (int)(padded / 16);
   const int work = n16 > n_rope_chunks * half_d ? n16 : n_rope_chunks * half_d;
-  store_blob_kernel<<<(work + 127) / 128, 128, 0, st>>>(blob, n16, reinterpret_cast<uint4*>(dst), n_rope_chunks, inv_freq, half_d,
-                                                         cs_table);
-  return cudaGetLastError();
+  return launch_pdl(store_blob_kernel, dim3((work + 127) / 128), dim3(128), 0, st, blob, n16, reinterpret_cast<uint4*>(dst), n_rope_chunks,
+                    inv_freq, half_d, cs_table);
 }
 
 }  // namespace kvb

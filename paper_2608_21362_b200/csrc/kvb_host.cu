@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "kvb_internal.h"
+#include "pdl.cuh"
 
 using namespace kvb;
 
@@ -228,6 +229,8 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, attention_tc_configure());
   const char* attn_env = getenv("KVB_ATTN");
   c->attn_legacy = attn_env && strcmp(attn_env, "mma") == 0;
+  const char* pdl_env = getenv("KVB_PDL");
+  pdl_enabled() = !(pdl_env && strcmp(pdl_env, "0") == 0);
   const char* desc_env = getenv("KVB_DESC");
   c->force_copy = desc_env && strcmp(desc_env, "copy") == 0;
   c->attn_mode = attn_env && strcmp(attn_env, "persistent") == 0 ? 1 : (attn_env && strcmp(attn_env, "onetile") == 0 ? 2 : 0);

@@ -11,6 +11,7 @@
 // selection, conflict-free shared-memory access, and the bitonic stages with stride < 32 done
 // in registers with shuffles.
 #include "kvb_internal.h"
+#include "pdl.cuh"
 
 namespace kvb {
 namespace {
@@ -79,6 +80,7 @@ __global__ void __launch_bounds__(kThreads, 1)
   __shared__ uint32_t s_hist[2][256];  // two buffers: one is cleared while the other is scanned
   __shared__ uint32_t s_pick[2];       // chosen bin, remaining need
 
+  pdl_wait();  // descriptors and deviation sums come from the kernels before this one
   const ReqDesc rq = reqs[blockIdx.x];
   const int T = rq.T, k = min(rq.k, T);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -345,8 +347,7 @@ cudaError_t launch_topk(const ReqDesc* reqs, int n_req, const SeamWindow* seams,
   int k_pad = 1;
   while (k_pad < max_k) k_pad <<= 1;
   const float inv_scale = (float)(1.0 / (1099511627776.0 * (double)n_terms));  // 2^-40 / n_terms
-  topk_kernel<<<n_req, kThreads, topk_smem(t_pad, k_pad), st>>>(reqs, seams, inv_scale, acc, t_pad, status);
-  return cudaGetLastError();
+  return launch_pdl(topk_kernel, dim3(n_req), dim3(kThreads), topk_smem(t_pad, k_pad), st, reqs, seams, inv_scale, acc, t_pad, status);
 }
 
 }  // namespace kvb
