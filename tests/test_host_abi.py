@@ -168,3 +168,82 @@ def test_wrong_chunk_size_is_rejected():
     t = _table()
     t.array[0].chunks[1].n_tokens = 64
     assert _st(t)[0] == B.KVB_ERR_BAD_TABLE
+
+
+# ---------------------------------------------------------------- property: the validator against a restatement of its rules
+def _expected_status(T, chunks, kv_ptr, fresh_ptr, need_payload):
+    """The header's table rules, written out again: first failing rule wins, in the order the library checks."""
+    C_ = 128
+    if T <= 0 or len(chunks) == 0:
+        return B.KVB_ERR_INVALID_ARG
+    if T % C_ != 0 or len(chunks) != T // C_:
+        return B.KVB_ERR_BAD_TABLE
+    if kv_ptr == 0 or fresh_ptr == 0:
+        return B.KVB_ERR_INVALID_ARG
+    if kv_ptr % 16 or fresh_ptr % 16:
+        return B.KVB_ERR_BAD_TABLE
+    for i, c in enumerate(chunks):
+        if c["n_tokens"] != C_ or c["new_pos"] != i * C_:
+            return B.KVB_ERR_BAD_TABLE
+        if not 0 <= c["mode"] <= 3:
+            return B.KVB_ERR_INVALID_ARG
+        if c["meta_fp16"] not in (0, 1):
+            return B.KVB_ERR_INVALID_ARG
+        if not 0 <= c["match"] <= 2:
+            return B.KVB_ERR_INVALID_ARG
+        if c["mode"] == 0:
+            continue
+        if c["orig_pos"] < 0 or c["orig_pos"] >= 1 << 24 or c["new_pos"] >= 1 << 24:
+            return B.KVB_ERR_BAD_TABLE
+        if c["match"] == 1 and c["orig_pos"] != c["new_pos"]:
+            return B.KVB_ERR_BAD_TABLE
+        if not need_payload:
+            continue
+        if c["k_codes"] == 0 or c["v_codes"] == 0:
+            return B.KVB_ERR_INVALID_ARG
+        if c["k_codes"] % 16 or c["v_codes"] % 16:
+            return B.KVB_ERR_BAD_TABLE
+        if c["mode"] != 1:
+            if c["k_meta"] == 0 or c["v_meta"] == 0:
+                return B.KVB_ERR_INVALID_ARG
+            if c["k_meta"] % 16 or c["v_meta"] % 16:
+                return B.KVB_ERR_BAD_TABLE
+    return B.KVB_OK
+
+
+def test_validator_agrees_with_the_stated_rules_on_random_tables():
+    hypothesis = pytest.importorskip("hypothesis")
+    from hypothesis import given, settings
+    from hypothesis import strategies as st
+
+    ptr = st.sampled_from([0, 0x1000, 0x1008, 0x2010, 0x7F00])
+    chunk = st.fixed_dictionaries({
+        "mode": st.sampled_from([0, 1, 2, 3, 3, 2, 4, -1]),
+        "match": st.sampled_from([0, 1, 2, 2, 2, 3]),
+        "meta_fp16": st.sampled_from([0, 0, 0, 1, 2]),
+        "n_tokens": st.sampled_from([128, 128, 128, 128, 64]),
+        "orig_pos": st.sampled_from([0, 128, 4096, (1 << 24) - 128, 1 << 24, -5]),
+        "pos_fault": st.sampled_from([0, 0, 0, 0, 0, 128, -128]),
+        "k_codes": ptr, "v_codes": ptr, "k_meta": ptr, "v_meta": ptr,
+    })
+
+    @settings(max_examples=300, deadline=None)
+    @given(st.lists(chunk, min_size=0, max_size=5), st.sampled_from([0, 0, 0, 128, -128, 64]), ptr, ptr, st.booleans())
+    def run(chunks, t_fault, kv_ptr, fresh_ptr, need_payload):
+        for i, c in enumerate(chunks):
+            c["new_pos"] = i * 128 + c["pos_fault"]
+        T = len(chunks) * 128 + t_fault
+        arr = (B.kvb_chunk * max(1, len(chunks)))()
+        for i, c in enumerate(chunks):
+            for name in ("orig_pos", "new_pos", "n_tokens", "mode", "match", "meta_fp16"):
+                setattr(arr[i], name, c[name])
+            for name in ("k_codes", "v_codes", "k_meta", "v_meta"):
+                setattr(arr[i], name, c[name] or None)
+        req = (B.kvb_request * 1)()
+        req[0].T, req[0].n_chunks, req[0].chunks = T, len(chunks), arr
+        req[0].kv_buf, req[0].fresh = kv_ptr or None, fresh_ptr or None
+        buf = C.create_string_buffer(512)
+        got = B.lib().kvb_validate(C.byref(MODEL), C.byref(LIMITS), req, 1, int(need_payload), buf, 512)
+        assert got == _expected_status(T, chunks, kv_ptr, fresh_ptr, need_payload), (buf.value, T, chunks)
+
+    run()
