@@ -176,7 +176,8 @@ int kvb_assemble_select(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const 
 /* Causal attention (Eq. 2) of the selected rows only.  q[r], out[r]: device,
  * [L][sel_capacity][Hq][d] in kv_dtype; row i belongs to position sel[i] and
  * attends keys 0..sel[i] of kv_buf; query head hq reads KV head hq/(Hq/Hkv).
- * Rows >= *n_sel are left untouched.  softmax in float32. */
+ * Rows >= *n_sel are left untouched.  softmax in float32.  q[r] must be
+ * 16-byte aligned, out[r] 32-byte aligned (KVB_ERR_BAD_TABLE otherwise). */
 int kvb_selective_attn(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_selection* sel,
                        const void* const* q, void* const* out, float softmax_scale, void* cuda_stream);
 

@@ -36,7 +36,8 @@ constexpr uint32_t kTileBytes = kRows * kD * 2;      // 32 KB: Q, K or V tile
 constexpr uint32_t kHalfBytes = kTileBytes / 2;      // one 64-element-wide TMA box of Q (128 rows)
 constexpr uint32_t kSubBytes = kSubKeys * kD * 2;    // 16 KB: one stream's K or V sub-block
 constexpr uint32_t kTmemCols = 256;                  // S/P: columns 0..127, O: columns 128..255
-constexpr uint32_t kWaitLimit = 1u << 24;
+constexpr uint32_t kWaitHintNs = 20000;              // per try; 2 us .. 200 us measured alike
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // a wait that lasts two seconds gives up
 constexpr float kLazyThreshold = 8.0f;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -51,23 +52,33 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One try with a suspend-time hint: the hardware parks the thread until the phase completes or the
+// hint (nanoseconds) runs out instead of returning at once.  Twelve warps per SM wait on barriers most
+// of the time; without the hint their re-issued tries crowd the queue that the MMA issue, the TMEM
+// loads and the global stores also go through (measured: +4 % on the whole kernel).
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kWaitHintNs)
       : "memory");
   return ok != 0;
 }
-// Bounded wait; also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait (kWaitLimitNs of wall time); also gives up as soon as another role has raised the abort flag.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  for (uint32_t i = 0; i < kWaitLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 255u) == 255u) {
-      if (*abort_flag) return false;
-      __nanosleep(128);
-    }
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) break;
   }
   *abort_flag = 1;
   return false;
@@ -200,6 +211,13 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
+}
+
+// One 32-byte store (the address must be 32-byte aligned).
+__device__ __forceinline__ void st_global_256(void* p, const uint32_t (&w)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]),
+               "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
 }
 
 template <int DT>
@@ -620,14 +638,14 @@ __global__ void __launch_bounds__(kThreads, 2)
         mbar_arrive(&bars.o_empty);
       }
       if (live_row) {
+        // 32-byte stores: what the epilogue costs goes with the number of store instructions (each
+        // touches 32 lines, one per row), not with their width
 #pragma unroll
-        for (int i = 0; i < 32; i += 8) {
-          uint4 w;
-          w.x = pack2<DT>(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-          w.y = pack2<DT>(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-          w.z = pack2<DT>(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-          w.w = pack2<DT>(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
-          *reinterpret_cast<uint4*>(orow + (c * 32 + i) * 2) = w;
+        for (int i = 0; i < 32; i += 16) {
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) w[j] = pack2<DT>(__uint_as_float(r[i + 2 * j]) * inv, __uint_as_float(r[i + 2 * j + 1]) * inv);
+          st_global_256(orow + (c * 32 + i) * 2, w);
         }
       }
     }

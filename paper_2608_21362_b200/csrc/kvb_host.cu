@@ -535,7 +535,8 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
     const kvb_selection& s = sel[r];
     if (!s.sel || !s.n_sel || s.sel_capacity <= 0 || !q[r] || !out[r])
       return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL sel / n_sel / q / out or empty capacity", r);
-    if (!aligned16(q[r]) || !aligned16(out[r])) return fail(c, KVB_ERR_BAD_TABLE, "request %d: q / out must be 16-byte aligned", r);
+    if (!aligned16(q[r]) || (reinterpret_cast<uintptr_t>(out[r]) & 31u) != 0)  // the output rows leave as 32-byte stores
+      return fail(c, KVB_ERR_BAD_TABLE, "request %d: q must be 16-byte aligned, out 32-byte aligned", r);
     ReqDesc d{};
     d.kv_buf = static_cast<const uint8_t*>(reqs[r].kv_buf);
     d.sel = s.sel;
