@@ -250,3 +250,34 @@ def test_empty_selection_and_wide_overlapping_seam_windows():
         assert int(sel.n_sel[0]) == r.plan.T  # three seams x 350 positions cover all 512
     finally:
         B.kvb_destroy(ctx)
+
+
+def test_attention_rejects_an_output_that_is_not_32_byte_aligned():
+    """Output rows leave the attention kernel as 32-byte stores; the call checks the base pointer on the
+    host and launches nothing when it is off (q only needs 16 bytes)."""
+    wl = synth.workload(0)
+    sh = wl.shape
+    reqs = prepare(wl)
+    (r,) = reqs
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, wl.select, use_oracle_buffer=False)
+        flat = torch.zeros(r.q.numel() + 8, dtype=r.q.dtype, device=DEV)
+        off = flat[8:].view(r.q.shape)  # 16 bytes past a 32-byte boundary
+        assert off.data_ptr() % 32 == 16
+        before = B.lib().kvb_launch_count(ctx)
+        st = B.kvb_selective_attn(ctx, tbl, sel, [r.q], [off], 0.1, check=False)
+        assert st == B.KVB_ERR_BAD_TABLE and B.lib().kvb_launch_count(ctx) == before
+        assert not flat.any()
+        q_off = torch.zeros(r.q.numel() + 8, dtype=r.q.dtype, device=DEV)[8:].view(r.q.shape)  # a 16-byte aligned q is fine
+        q_off.copy_(r.q)
+        out = torch.zeros_like(r.q)
+        B.kvb_selective_attn(ctx, tbl, sel, [q_off], [out], 1.0 / math.sqrt(sh.d))
+        B.kvb_last_status(ctx)
+        ref = torch.zeros_like(r.q)
+        B.kvb_selective_attn(ctx, tbl, sel, [r.q], [ref], 1.0 / math.sqrt(sh.d))
+        B.kvb_last_status(ctx)
+        assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
+    finally:
+        B.kvb_destroy(ctx)
