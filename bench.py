@@ -461,10 +461,10 @@ def main():
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the committed ncu captures
     # (profiles/cfg1_launches_and_kernels.md, profiles/cfg2_kernels.md); null where none was taken
     ncu_traffic = {
-        ("cfg1_qwen3b_2k_int8", "selective_attn"): 208.2e6, ("cfg1_qwen3b_2k_int8", "assemble"): 67.6e6,
-        ("cfg1_qwen3b_2k_int8", "assemble_select"): 126.6e6,
-        ("cfg1_qwen3b_2k_int8", "deviation_topk"): 154.2e6, ("cfg2_long_int4_8k", "selective_attn"): 720.2e6,
-        ("cfg2_long_int4_8k", "assemble_select"): 648.3e6,
+        ("cfg1_qwen3b_2k_int8", "selective_attn"): 211.9e6, ("cfg1_qwen3b_2k_int8", "assemble"): 67.6e6,
+        ("cfg1_qwen3b_2k_int8", "assemble_select"): 125.6e6,
+        ("cfg1_qwen3b_2k_int8", "deviation_topk"): 154.2e6, ("cfg2_long_int4_8k", "selective_attn"): 730.0e6,
+        ("cfg2_long_int4_8k", "assemble_select"): 646.8e6,
         ("cfg2_long_int4_8k", "assemble"): 381.0e6, ("cfg2_long_int4_8k", "deviation_topk"): 608.2e6,
     }
     roof.update({"kernel": top, "traffic": ncu_traffic.get((wl.name, top)), "peak_source": "%s (%s)" % (peaks["source"], "sustained" if (top == "selective_attn" and long_run) else "burst/copy"),
