@@ -125,3 +125,52 @@ def test_fused_rejects_what_either_call_rejects():
         assert B.kvb_launch_count(ctx) == before
     finally:
         B.kvb_destroy(ctx)
+
+
+@pytest.mark.parametrize("seed", [1, 3, 8, 13])
+def test_random_ragged_batches_through_the_one_pass_path_and_attention(seed):
+    """Seeded random batches: head counts, layers, dtype, request lengths, chunk modes and original
+    positions (aligned, unaligned, unmoved), selection ratio (0 and 1 included), seam windows, which of
+    K / V is compared and attention sinks are all drawn; stitch, selection and attention are checked
+    against the oracle."""
+    import math
+
+    from test_gpu_parity import check_attention
+
+    M = synth
+    rng = np.random.default_rng(1000 + seed)
+    Hkv, rep, dt = int(rng.choice([1, 2, 4, 8])), int(rng.choice([1, 2, 4, 8])), str(rng.choice(["bf16", "fp16"]))
+    sh = M.Shape(L=int(rng.integers(1, 4)), Hq=Hkv * rep, Hkv=Hkv, kv_dtype=dt)
+    plans = []
+    for _ in range(int(rng.integers(1, 5))):
+        nch = int(rng.integers(1, 11))
+        modes = rng.choice([M.MODE_FRESH, M.MODE_FP16, M.MODE_INT8, M.MODE_INT4], size=nch, p=[0.25, 0.25, 0.3, 0.2])
+        origs = [int(rng.integers(0, (1 << 24) - 128)) if rng.random() < 0.7 else int(rng.integers(0, 64)) * 128 for _ in range(nch)]
+        origs = [i * sh.C if rng.random() < 0.2 else o for i, o in enumerate(origs)]
+        plans.append(M._request(nch * sh.C, sh.C, list(modes), origs))
+    sp = M.SelectPlan(ratio=float(rng.choice([0.0, 0.05, 0.15, 0.5, 1.0])), seam_before=int(rng.choice([0, 4, 16, 40])),
+                      seam_after=int(rng.choice([0, 8, 16])), which=int(rng.choice([1, 2, 3])))
+    sinks = int(rng.choice([0, 0, 4]))
+    wl = M.Workload("rand", 1000 + seed, sh, plans, sp)
+    reqs = prepare(wl)
+    ctx = B.create_for_shape(sh, 0, max_requests=len(reqs))
+    try:
+        tbl, sel, ks = run_fused(ctx, wl, reqs, sp, sink_tokens=sinks)
+        for r in reqs:
+            kv_o, exact = oracle_stitch(sh, r)
+            check_assembled(sh, r, helpers.bits_of(r.kv_buf), exact, kv_o)
+        if sinks == 0:
+            check_selection(sh, reqs, sel, ks, sp)
+        qs = [(torch.randn(sh.L, sel.sel[i].numel(), sh.Hq, sh.d, device=DEV, generator=torch.Generator(DEV).manual_seed(seed * 10 + i)) / math.sqrt(sh.d)).to(r.fresh.dtype)
+              for i, r in enumerate(reqs)]
+        outs = [torch.zeros_like(q) for q in qs]
+        B.kvb_selective_attn(ctx, tbl, sel, qs, outs, 1.0 / math.sqrt(sh.d))
+        B.kvb_last_status(ctx)
+        for i, r in enumerate(reqs):
+            n = int(sel.n_sel[i])
+            r.q = qs[i]
+            if n:
+                check_attention(sh, r, sel.sel[i].cpu().numpy()[:n], outs[i], None, None)
+            assert not outs[i][:, n:].any()
+    finally:
+        B.kvb_destroy(ctx)

@@ -440,3 +440,29 @@ def test_rejected_calls_launch_nothing():
         B.kvb_destroy(ctx)
     with pytest.raises(B.KvbError):
         B.create_for_shape(synth.Shape(d=64))  # head_dim the kernels are not built for
+
+
+# ------------------------------------------------------------------------------- shape corners
+@pytest.mark.parametrize("Hkv,Hq,kv_dtype", [(1, 16, "bf16"), (16, 16, "fp16"), (16, 64, "bf16"), (8, 128, "bf16"), (4, 16, "fp16")])
+def test_whole_path_at_the_corners_of_the_supported_shapes(Hkv, Hq, kv_dtype):
+    """Stitch, deviation + selection and attention against the oracle at the ends of the supported head
+    counts (1 and 16 KV heads; 1, 4 and 16 query heads per KV head), every mode in one request."""
+    sh = synth.Shape(L=2, Hq=Hq, Hkv=Hkv, kv_dtype=kv_dtype)
+    modes = [synth.MODE_INT8, synth.MODE_INT4, synth.MODE_FRESH, synth.MODE_FP16, synth.MODE_INT8]
+    wl = synth.Workload("corner", 100 + 17 * Hkv + Hq, sh, [synth._request(640, sh.C, modes, [384, 7, 0, 1 << 18, 512])],
+                        synth.SelectPlan(ratio=0.15, seam_before=8, seam_after=8))
+    reqs = prepare(wl)
+    (r,) = reqs
+    ctx = _ctx(sh)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        kv_o, exact = oracle_stitch(sh, r)
+        check_assembled(sh, r, helpers.bits_of(r.kv_buf), exact, kv_o)
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, wl.select, use_oracle_buffer=False)
+        check_selection(sh, reqs, sel, ks, wl.select)
+        n = int(sel.n_sel[0])
+        (out,) = run_attention(ctx, sh, reqs, tbl, sel)
+        check_attention(sh, r, sel.sel[0].cpu().numpy()[:n], out, None, None)
+        assert not out[:, n:].any()
+    finally:
+        B.kvb_destroy(ctx)
