@@ -272,6 +272,14 @@ const char* kvb_status_string(int status);
 /* Number of kernels this context has launched so far. */
 int64_t kvb_launch_count(kvb_ctx* ctx);
 
+/* Self-test of the error path of a stuck barrier wait: launches one warp that
+ * waits, with the attention kernel's own bounded wait, on a barrier that
+ * nothing ever completes.  After limit_ms (1..1000) the wait gives up, the
+ * kernel returns and sets status bit 0x1; the next kvb_last_status reports
+ * KVB_ERR_DEVICE_STATUS and the context stays usable.  Asynchronous on the
+ * stream like the data-path calls. */
+int kvb_selftest_wait_timeout(kvb_ctx* ctx, int limit_ms, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -299,6 +299,13 @@ def kvb_launch_count(ctx) -> int:
     return int(lib().kvb_launch_count(ctx))
 
 
+def kvb_selftest_wait_timeout(ctx, limit_ms: int, stream=None, check: bool = True) -> int:
+    L = lib()
+    L.kvb_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int, C.c_void_p]
+    st = L.kvb_selftest_wait_timeout(ctx, limit_ms, _stream(stream))
+    return _check(ctx, st) if check else st
+
+
 # ------------------------------------------------------------------ small conveniences over the entry points
 def create_for_shape(sh, device: int = 0, max_requests: int = 64, max_chunks_total: int = 8192,
                      max_tokens_total: int = 1 << 20):

@@ -70,18 +70,21 @@ __device__ __forceinline__ unsigned long long global_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-// Bounded wait (kWaitLimitNs of wall time); also gives up as soon as another role has raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// Bounded wait (limit_ns of wall time); also gives up as soon as another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait_ns(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag, unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitLimitNs) break;
+    if (global_ns() - t0 > limit_ns) break;
   }
   *abort_flag = 1;
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  return mbar_wait_ns(bar, parity, abort_flag, kWaitLimitNs);
 }
 
 // ---- TMA
@@ -663,6 +666,21 @@ __global__ void __launch_bounds__(kThreads, 2)
   if (tid == 0 && s_abort) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
 }
 
+// The error path of a stuck wait, on its own: a barrier that expects one arrival and gets none.
+__global__ void wait_selftest_kernel(uint32_t* __restrict__ status, unsigned long long limit_ns) {
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t s_abort;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  mbar_wait_ns(&bar, 0, &s_abort, limit_ns);
+  __syncthreads();
+  if (threadIdx.x == 0 && s_abort) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
+}
+
 constexpr size_t kSmemBytes = 3 * kTileBytes + 1024;
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -715,6 +733,11 @@ int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity
       return 3;
   }
   return 0;
+}
+
+cudaError_t launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, cudaStream_t st) {
+  wait_selftest_kernel<<<1, 32, 0, st>>>(status, limit_ns);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,

@@ -189,6 +189,17 @@ int kvb_validate(const kvb_model_desc* model, const kvb_limits* limits, const kv
 const char* kvb_last_error(kvb_ctx* c) { return c ? c->err : "NULL context"; }
 int64_t kvb_launch_count(kvb_ctx* c) { return c ? c->launches : 0; }
 
+int kvb_selftest_wait_timeout(kvb_ctx* c, int limit_ms, void* cuda_stream) {
+  if (!c) return KVB_ERR_INVALID_ARG;
+  if (limit_ms < 1 || limit_ms > 1000) return fail(c, KVB_ERR_INVALID_ARG, "limit_ms must be in 1..1000");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+  KVB_CUDA(c, launch_wait_selftest(c->status_dev, (unsigned long long)limit_ms * 1000000ull, st));
+  c->last_stream = st;
+  c->launches += 1;
+  return KVB_OK;
+}
+
 int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb_limits* limits) {
   if (!out || !model || !limits) return KVB_ERR_INVALID_ARG;
   *out = nullptr;

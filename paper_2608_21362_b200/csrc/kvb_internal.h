@@ -89,6 +89,8 @@ cudaError_t launch_attention_mma(const ReqDesc* reqs, int n_req, int total_tiles
 cudaError_t attention_mma_configure();
 
 cudaError_t attention_tc_configure();
+// One warp waits on a barrier nothing completes; gives up after limit_ns and raises DEV_STATUS_WAIT_TIMEOUT.
+cudaError_t launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, cudaStream_t st);
 // Encodes the request's two TMA tensor maps (Q, KV) into out[0..255]; returns 0 on success.
 int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity, const void* kv_buf, int T, void* out);
 // persistent: 2 CTAs per SM drawing tiles from *tile_counter (a zeroed device word), else one tile per CTA;

@@ -281,3 +281,37 @@ def test_attention_rejects_an_output_that_is_not_32_byte_aligned():
         assert torch.equal(out.view(torch.int16), ref.view(torch.int16))
     finally:
         B.kvb_destroy(ctx)
+
+
+def test_a_barrier_wait_that_cannot_complete_gives_up_and_is_reported():
+    """The attention kernel's waits are bounded by wall time.  The library's self-test runs that wait on
+    a barrier nothing arrives at: the kernel must return after the limit, raise status bit 0x1, and
+    leave the context fit for the next call."""
+    import time
+
+    wl = synth.workload(0)
+    sh = wl.shape
+    reqs = prepare(wl)
+    (r,) = reqs
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        assert B.kvb_selftest_wait_timeout(ctx, 0, check=False) == B.KVB_ERR_INVALID_ARG
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        B.kvb_selftest_wait_timeout(ctx, 30)
+        with pytest.raises(B.KvbError) as ei:
+            B.kvb_last_status(ctx)  # synchronises
+        dt = time.perf_counter() - t0
+        assert ei.value.status == B.KVB_ERR_DEVICE_STATUS and "0x1" in str(ei.value) and "wait" in str(ei.value)
+        assert 0.03 <= dt < 1.0, dt
+        assert B.kvb_last_status(ctx) == B.KVB_OK  # reported once
+        # the context still works
+        tbl = run_assemble(ctx, reqs)
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, wl.select, use_oracle_buffer=False)
+        out = torch.zeros_like(r.q)
+        B.kvb_selective_attn(ctx, tbl, sel, [r.q], [out], 1.0 / math.sqrt(sh.d))
+        assert B.kvb_last_status(ctx) == B.KVB_OK
+        n = int(sel.n_sel[0])
+        check_attention(sh, r, sel.sel[0].cpu().numpy()[:n], out, None, None)
+    finally:
+        B.kvb_destroy(ctx)
