@@ -267,7 +267,7 @@ __device__ __forceinline__ NextTile decode_next_tile(unsigned int& drawn, unsign
       const long long lin_ll = drawn;
       if (lin_ll >= (long long)total_tiles * per_tile) break;
       const int lin = (int)lin_ll;
-      drawn = PERSISTENT ? atomicAdd(tile_counter, 1u) : kNoTile;
+      drawn = PERSISTENT ? gridDim.x + atomicAdd(tile_counter, 1u) : kNoTile;  // the first gridDim.x tiles went by block index
       int lo = 0, hi = n_req - 1;
       while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
@@ -338,7 +338,8 @@ __global__ void __launch_bounds__(kThreads, 2)
   if (tid == 0) {
     pdl_wait();  // descriptors, tensor maps and the tile counter come from the kernel before this one; the
                  // other roles touch global memory only after this thread has published a tile
-    drawn = PERSISTENT ? atomicAdd(tile_counter, 1u) : blockIdx.x;
+    drawn = blockIdx.x;  // a CTA's first tile is its block index (the grid never exceeds the tile count): no
+                         // round trip to the counter in front of the kernel's first loads
   }
   auto decode_next = [&]() { return decode_next_tile<PERSISTENT>(drawn, tile_counter, reqs, maps, n_req, total_tiles, per_tile, TOK, m.Hkv); };
   NextTile next;
