@@ -77,8 +77,14 @@ def check_assembled(sh, req, kv_gpu_bits, exact, kv_oracle_bits):
         err = np.abs(g[:, :, sl] - y)
         worst = float((err / bound).max())
         assert worst <= 1.0, "chunk at %d (mode %d): error %.3g x bound" % (ck.plan.new_pos, ck.plan.mode, worst)
+    # Beyond the tolerance: how often the two 16-bit roundings coincide.  The GPU rounds a float32 result
+    # whose error e is a few 2^-24 of the chunk's magnitude M, the oracle rounds the exact value; they
+    # differ when y lies within e of a rounding boundary, i.e. with probability ~ 2e / ulp16(y)
+    # = c * 2^-23 * (M/|y|) / 2^-p (p = 8 bits for bf16, 11 for fp16; c ~ 2..3, mean M/|y| ~ 3):
+    # about 3e-4 in bf16 and 2e-3 in fp16 (measured: up to 2.2e-3 on int4 keys in fp16).
     agree = float(np.mean(kv_gpu_bits == kv_oracle_bits))
-    assert agree > 0.999, "only %.5f of stored values equal the oracle's rounding bit for bit" % agree
+    floor = 0.999 if sh.kv_dtype == "bf16" else 0.995
+    assert agree > floor, "only %.5f of stored values equal the oracle's rounding bit for bit" % agree
     return agree
 
 
