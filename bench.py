@@ -270,6 +270,7 @@ def main():
     ap.add_argument("--workload", default="cfg1", choices=sorted(WORKLOADS))
     ap.add_argument("--replicas", type=int, default=0, help="independent copies rotated through (0 = auto)")
     ap.add_argument("--batch", type=int, default=1, help="requests per step: the workload's request list repeated this many times")
+    ap.add_argument("--requests", type=int, default=0, help="cfg4 only: the ragged batch's first N requests instead of all 32")
     ap.add_argument("--path", default="one-pass", choices=["one-pass", "two-call"], help="kvb_assemble_select, or kvb_assemble + kvb_deviation_topk")
     ap.add_argument("--meta-fp16", action="store_true", help="cached chunks carry compact (binary16) scale/min pairs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -278,7 +279,11 @@ def main():
     args.warmup = max(args.warmup, 3)
     global ONE_PASS
     ONE_PASS = args.path == "one-pass"
-    wl = synth.workload(WORKLOADS[args.workload])
+    if args.requests > 0 and args.workload != "cfg4":
+        ap.error("--requests applies to --workload cfg4")
+    wl = synth.workload(WORKLOADS[args.workload], args.requests if args.requests > 0 else None)
+    if args.requests > 0:  # a reduced ragged batch (profiling under a memory limit); not the workload the benchmark spec names
+        wl = synth.Workload("%s_first%d" % (wl.name, args.requests), wl.seed, wl.shape, wl.requests, wl.select, wl.sigma_bulk, wl.sigma_seam, wl.seam_tokens)
     if args.batch > 1:
         wl = synth.Workload("%s_x%d" % (wl.name, args.batch), wl.seed, wl.shape, wl.requests * args.batch, wl.select, wl.sigma_bulk, wl.sigma_seam, wl.seam_tokens)
     if args.impl == "reference":
