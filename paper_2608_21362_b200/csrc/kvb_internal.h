@@ -60,10 +60,12 @@ struct ModelDims {
 };
 
 // ---- launchers (each defined next to its kernel) ----
-// Tables of at most kDescBlobBytes go to the arena as a kernel argument (csrc/desc_store.cu); the
+// Tables of at most kDescBlobBytes go to the arena as a kernel argument (csrc/desc_store.cu; two
+// argument sizes, 3840 and 16384 bytes, so a small call does not pay for a large argument); the
 // chunk descriptors, if any, must be at the start of the bytes, and n_rope_chunks > 0 also fills
 // cs_table[n_rope_chunks][half_d] from their delta_pos.
-constexpr size_t kDescBlobBytes = 3840;
+constexpr size_t kDescBlobSmall = 3840;
+constexpr size_t kDescBlobBytes = 16384;
 cudaError_t launch_store_blob(const void* host_bytes, size_t bytes, uint8_t* dst, int n_rope_chunks, const double* inv_freq,
                               int half_d, float2* cs_table, cudaStream_t st);
 // launch_assemble: acc != NULL fuses the deviation sums (which: bit 0 keys, bit 1 values) into the stitch.
