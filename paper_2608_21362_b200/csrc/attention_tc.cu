@@ -9,9 +9,12 @@
 //     P = exp2(scale*S - m)  by 128 threads, one TMEM lane (row) each, written back over S as bf16
 //     O += P V    tcgen05.mma, P from TMEM, V from shared memory (MN-major), O in TMEM
 // Tiles are fetched by TMA (cp.async.bulk.tensor) with mbarrier completion.  Warp roles: warp 0
-// lane 0 issues TMA, warp 1 lane 0 issues MMAs (and owns the TMEM allocation), warps 2-5 do the
-// softmax and the epilogue.  Each CTA uses 256 TMEM columns and 96 KB of shared memory so that two
-// CTAs share an SM: one CTA's softmax overlaps the other's MMAs.
+// lane 0 issues TMA; warp 1 issues the MMAs (and owns the TMEM allocation): the whole warp runs the
+// issue loop so that its descriptor arithmetic stays warp-uniform, and one lane chosen by elect.sync
+// executes each tcgen05.mma / tcgen05.commit (a microbenchmark puts one thread's issue interval at
+// 36 cycles this way against 51 from inside an `if (lane == 0)` region); warps 2-5 do the softmax
+// and the epilogue.  Each CTA uses 256 TMEM columns and 96 KB of shared memory so that two CTAs
+// share an SM: one CTA's softmax overlaps the other's MMAs.
 //
 // The running maximum is lazy: the reference m only moves when a block's maximum exceeds it by
 // more than 8 (a factor 256), in which case the O rows in TMEM are rescaled; P stays within
@@ -108,17 +111,17 @@ __device__ __forceinline__ void tensormap_acquire(const CUtensorMap* map) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+  asm volatile("{\n .reg .pred e;\n elect.sync _|e, 0xffffffff;\n @e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n @e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+      "{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.ne.b32 p, %4, 0;\n @e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -126,13 +129,13 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
 // thread's instruction count matters).
 __device__ __forceinline__ void mma_ss_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.eq.b32 p, 0, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
+      "{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.eq.b32 p, 0, 0;\n @e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(d_tmem),
       "l"(a_desc), "l"(b_desc), "r"(idesc)
       : "memory");
 }
 __device__ __forceinline__ void mma_ts_acc(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc) {
   asm volatile(
-      "{\n .reg .pred p;\n setp.eq.b32 p, 0, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
+      "{\n .reg .pred p, e;\n elect.sync _|e, 0xffffffff;\n setp.eq.b32 p, 0, 0;\n @e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}" ::"r"(d_tmem),
       "r"(a_tmem), "l"(b_desc), "r"(idesc)
       : "memory");
 }
@@ -440,7 +443,7 @@ __global__ void __launch_bounds__(kThreads, 2)
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    {  // the whole warp runs the loop (its address arithmetic stays warp-uniform); one elected lane issues
       const uint32_t idesc_s = instr_desc<DT>(kSubKeys, false);
       const uint32_t idesc_pv = instr_desc<DT>(kD, true);
       const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
@@ -489,7 +492,8 @@ __global__ void __launch_bounds__(kThreads, 2)
         ok = mbar_wait(&bars.tile_full[slot], (n >> 1) & 1, abort_flag);
         if (!ok) break;
         const int nsb = s_tiles[slot].nsb;
-        mbar_arrive(&bars.tile_empty[slot]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.tile_empty[slot]);
         if (nsb == 0) break;
         ok = mbar_wait(&bars.q_full, n & 1, abort_flag);
         if (!ok) break;
