@@ -138,7 +138,10 @@ typedef struct {
 } kvb_selection;
 
 /* Creates a context on `device` (a CUDA ordinal).  Allocates the descriptor
- * arena (pinned host + device) and the deviation scratch for the given limits. */
+ * arena (pinned host + device) and the deviation scratch for the given limits.
+ * KVB_ERR_UNSUPPORTED for shapes the kernels are not built for (d, chunk_tokens
+ * other than 128, int4_group other than 32, head counts that are not powers of
+ * two up to 16, L > 65535) and for limits beyond 2^31-1 tokens per call. */
 int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb_limits* limits);
 int kvb_destroy(kvb_ctx* ctx);
 
@@ -177,7 +180,8 @@ int kvb_assemble_select(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const 
  * [L][sel_capacity][Hq][d] in kv_dtype; row i belongs to position sel[i] and
  * attends keys 0..sel[i] of kv_buf; query head hq reads KV head hq/(Hq/Hkv).
  * Rows >= *n_sel are left untouched.  softmax in float32.  q[r] must be
- * 16-byte aligned, out[r] 32-byte aligned (KVB_ERR_BAD_TABLE otherwise). */
+ * 16-byte aligned, out[r] 32-byte aligned (KVB_ERR_BAD_TABLE otherwise).
+ * reqs[r].fresh is not read and may be NULL. */
 int kvb_selective_attn(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_selection* sel,
                        const void* const* q, void* const* out, float softmax_scale, void* cuda_stream);
 
@@ -192,7 +196,8 @@ int kvb_patch(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_select
  * Eq. 7): importance[r][c] = 1/(L*H*C) * sum over layers, KV heads and the C
  * tokens of chunk c of ||k||_2, read from the stitched kv_buf (a rotation
  * leaves the norms unchanged).  importance: host array of n_req device
- * pointers, each to n_chunks float32 values. */
+ * pointers, each to n_chunks float32 values.  reqs[r].fresh is not read and
+ * may be NULL. */
 int kvb_chunk_importance(kvb_ctx* ctx, const kvb_request* reqs, int n_req, float* const* importance,
                          void* cuda_stream);
 
@@ -239,9 +244,12 @@ int kvb_quantize_chunk_ex(kvb_ctx* ctx, const void* x, int is_value, int bits, i
  *   delta          device, [T] float32, written
  *   T              1 .. 16384; larger returns KVB_ERR_WORKSPACE (use a context)
  *   which          bit 0 keys, bit 1 values
- * Asynchronous on cuda_stream.  The first call on a device resolves the array's
- * device address (cudaGetSymbolAddress) and should come before any stream
- * capture.  All calls share the one array, which keeps the previous call's
+ *   model          L <= 65535 (KVB_ERR_UNSUPPORTED beyond), d = 128
+ * Asynchronous on cuda_stream.  The call makes `device` current while it
+ * launches and restores the caller's current device before it returns.  The
+ * first call on a device resolves the array's device address
+ * (cudaGetSymbolAddress) and should come before any stream capture; first
+ * calls from several host threads at once are safe.  All calls share the one array, which keeps the previous call's
  * contents (this call clears what it sums into): two calls whose GPU work
  * overlaps, e.g. on different streams, race on it. */
 int kvb_deviation_static(int device, const kvb_model_desc* model, const void* kv_buf, const void* fresh, int T,
@@ -271,6 +279,18 @@ const char* kvb_last_error(kvb_ctx* ctx);
 const char* kvb_status_string(int status);
 /* Number of kernels this context has launched so far. */
 int64_t kvb_launch_count(kvb_ctx* ctx);
+
+/* Test hook (the paper has no counterpart): switches one of the context's
+ * cross-check paths on (1) or off (0) for its later calls.  Keys:
+ *   "dependent_launch"            default 1; 0 launches the kernel chain without
+ *                                 programmatic dependent launch
+ *   "descriptor_copy"             default 0; 1 sends every descriptor table through
+ *                                 the pinned staging ring and cudaMemcpyAsync
+ *   "attention_one_tile_per_cta"  default 0; 1 runs kvb_selective_attn with one tile
+ *                                 per CTA instead of persistent CTAs
+ * Every setting computes the same results; the tests compare them bit for bit.
+ * Unknown key or value: KVB_ERR_INVALID_ARG. */
+int kvb_set_debug_option(kvb_ctx* ctx, const char* key, int value);
 
 /* Self-test of the error path of a stuck barrier wait: launches one warp that
  * waits, with the attention kernel's own bounded wait, on a barrier that

@@ -299,6 +299,13 @@ def kvb_launch_count(ctx) -> int:
     return int(lib().kvb_launch_count(ctx))
 
 
+def kvb_set_debug_option(ctx, key: str, value: int, check: bool = True) -> int:
+    L = lib()
+    L.kvb_set_debug_option.argtypes = [C.c_void_p, C.c_char_p, C.c_int]
+    st = L.kvb_set_debug_option(ctx, key.encode(), int(value))
+    return _check(ctx, st) if check else st
+
+
 def kvb_selftest_wait_timeout(ctx, limit_ms: int, stream=None, check: bool = True) -> int:
     L = lib()
     L.kvb_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int, C.c_void_p]

@@ -515,19 +515,19 @@ cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const doubl
 }
 
 cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
-                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, cudaStream_t st) {
+                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, bool pdl, cudaStream_t st) {
   const unsigned grid = (unsigned)n_chunks * m.L * 2 * assemble_split(m.Hkv);
   const bool dev = acc != nullptr && (which & 3);
   if (m.dtype == KVB_DT_BF16) {
     if (dev)
-      return launch_pdl(assemble_kernel<__nv_bfloat16, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
+      return launch_pdl(pdl, assemble_kernel<__nv_bfloat16, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
     else
-      return launch_pdl(assemble_kernel<__nv_bfloat16, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
+      return launch_pdl(pdl, assemble_kernel<__nv_bfloat16, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
   } else {
     if (dev)
-      return launch_pdl(assemble_kernel<__half, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
+      return launch_pdl(pdl, assemble_kernel<__half, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
     else
-      return launch_pdl(assemble_kernel<__half, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
+      return launch_pdl(pdl, assemble_kernel<__half, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
   }
   return cudaGetLastError();
 }

@@ -747,22 +747,22 @@ cudaError_t launch_wait_selftest(uint32_t* status, unsigned long long limit_ns, 
 
 cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,
                                 float scale, uint32_t* status, unsigned int* tile_counter, int n_sm, bool persistent,
-                                cudaStream_t st) {
+                                bool pdl, cudaStream_t st) {
   const long long work = (long long)total_tiles * m.Hkv * m.L;
   const float scale_log2 = scale * 1.4426950408889634f;
   const CUtensorMap* mp = static_cast<const CUtensorMap*>(maps);
   if (persistent) {  // two CTAs per SM; each takes tiles from *tile_counter (zero at launch) until they run out
     const unsigned grid = (unsigned)(work < 2LL * n_sm ? work : 2LL * n_sm);
     if (m.dtype == KVB_DT_BF16)
-      return launch_pdl(attn_tc_kernel<KVB_DT_BF16, true>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(pdl, attn_tc_kernel<KVB_DT_BF16, true>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
     else
-      return launch_pdl(attn_tc_kernel<KVB_DT_F16, true>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(pdl, attn_tc_kernel<KVB_DT_F16, true>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
   } else {
     const unsigned grid = (unsigned)work;
     if (m.dtype == KVB_DT_BF16)
-      return launch_pdl(attn_tc_kernel<KVB_DT_BF16, false>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(pdl, attn_tc_kernel<KVB_DT_BF16, false>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
     else
-      return launch_pdl(attn_tc_kernel<KVB_DT_F16, false>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
+      return launch_pdl(pdl, attn_tc_kernel<KVB_DT_F16, false>, dim3(grid), dim3(kThreads), kSmemBytes, st, reqs, mp, n_req, total_tiles, m, scale_log2, status, tile_counter);
   }
   return cudaGetLastError();
 }

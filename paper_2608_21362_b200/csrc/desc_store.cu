@@ -39,23 +39,23 @@ __global__ void __launch_bounds__(128)
 
 template <size_t BYTES>
 cudaError_t launch_sized(const void* host_bytes, size_t bytes, uint8_t* dst, int n_rope_chunks, const double* inv_freq, int half_d,
-                         float2* cs_table, cudaStream_t st) {
+                         float2* cs_table, bool pdl, cudaStream_t st) {
   DescBlob<BYTES> blob;
   const size_t padded = (bytes + 15) & ~(size_t)15;
   memcpy(&blob, host_bytes, bytes);
   if (padded > bytes) memset(reinterpret_cast<uint8_t*>(&blob) + bytes, 0, padded - bytes);
   const int n16 = (int)(padded / 16);
   const int work = n16 > n_rope_chunks * half_d ? n16 : n_rope_chunks * half_d;
-  return launch_pdl(store_blob_kernel<BYTES>, dim3((work + 127) / 128), dim3(128), 0, st, blob, n16, reinterpret_cast<uint4*>(dst),
+  return launch_pdl(pdl, store_blob_kernel<BYTES>, dim3((work + 127) / 128), dim3(128), 0, st, blob, n16, reinterpret_cast<uint4*>(dst),
                     n_rope_chunks, inv_freq, half_d, cs_table);
 }
 
 }  // namespace
 
 cudaError_t launch_store_blob(const void* host_bytes, size_t bytes, uint8_t* dst, int n_rope_chunks, const double* inv_freq,
-                              int half_d, float2* cs_table, cudaStream_t st) {
-  if (bytes <= kDescBlobSmall) return launch_sized<kDescBlobSmall>(host_bytes, bytes, dst, n_rope_chunks, inv_freq, half_d, cs_table, st);
-  if (bytes <= kDescBlobBytes) return launch_sized<kDescBlobBytes>(host_bytes, bytes, dst, n_rope_chunks, inv_freq, half_d, cs_table, st);
+                              int half_d, float2* cs_table, bool pdl, cudaStream_t st) {
+  if (bytes <= kDescBlobSmall) return launch_sized<kDescBlobSmall>(host_bytes, bytes, dst, n_rope_chunks, inv_freq, half_d, cs_table, pdl, st);
+  if (bytes <= kDescBlobBytes) return launch_sized<kDescBlobBytes>(host_bytes, bytes, dst, n_rope_chunks, inv_freq, half_d, cs_table, pdl, st);
   return cudaErrorInvalidValue;
 }
 

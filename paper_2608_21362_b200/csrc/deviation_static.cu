@@ -11,6 +11,8 @@
 // only where its scratch lives differs.
 #include <stdint.h>
 
+#include <atomic>
+
 #include "kvb_internal.h"
 
 using namespace kvb;
@@ -27,7 +29,22 @@ static_assert(sizeof(ReqDesc) <= kDescWords * sizeof(unsigned long long), "descr
 
 // Device address of g_static_scratch per GPU.  In host code the array's name is only a handle for
 // the runtime, not an address a kernel can use, so it is resolved once per device.
-void* g_scratch_addr[kMaxDevices] = {nullptr};
+// Several host threads may make their first call at once: each resolves the same address and the
+// atomic store publishes it.
+std::atomic<void*> g_scratch_addr[kMaxDevices];
+
+// Makes `device` current for the scope and puts the caller's current device back afterwards.
+struct DeviceScope {
+  int prev = -1;
+  bool ok = false;
+  explicit DeviceScope(int device) {
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    ok = cudaSetDevice(device) == cudaSuccess;
+  }
+  ~DeviceScope() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
 
 __global__ void store_desc_kernel(ReqDesc d, ReqDesc* dst) { *dst = d; }
 
@@ -46,20 +63,21 @@ extern "C" int kvb_deviation_static(int device, const kvb_model_desc* model, con
   if (device < 0 || device >= kMaxDevices) return KVB_ERR_INVALID_ARG;
   const kvb_model_desc& m = *model;
   const bool pow2_h = m.Hkv > 0 && (m.Hkv & (m.Hkv - 1)) == 0 && m.Hkv <= 16;
-  if (m.L <= 0 || m.d != 128 || !pow2_h || (m.kv_dtype != KVB_DT_F16 && m.kv_dtype != KVB_DT_BF16))
-    return KVB_ERR_UNSUPPORTED;
+  if (m.L <= 0 || m.L > 65535 || m.d != 128 || !pow2_h || (m.kv_dtype != KVB_DT_F16 && m.kv_dtype != KVB_DT_BF16))
+    return KVB_ERR_UNSUPPORTED;  // L is a grid y dimension
   if (T <= 0) return KVB_ERR_INVALID_ARG;
   if (T > kStaticMaxTokens) return KVB_ERR_WORKSPACE;  // beyond the static scratch: use the context API
   if ((reinterpret_cast<uintptr_t>(kv_buf) | reinterpret_cast<uintptr_t>(fresh)) & 15u) return KVB_ERR_BAD_TABLE;
 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (cudaSetDevice(device) != cudaSuccess) return KVB_ERR_NO_DEVICE;
-  if (!g_scratch_addr[device]) {  // first call on this device: resolve the symbol (do this before any stream capture)
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return KVB_ERR_CUDA;
-    g_scratch_addr[device] = p;
+  DeviceScope scope(device);
+  if (!scope.ok) return KVB_ERR_NO_DEVICE;
+  void* resolved = g_scratch_addr[device].load(std::memory_order_acquire);
+  if (!resolved) {  // first call on this device: resolve the symbol (do this before any stream capture)
+    if (cudaGetSymbolAddress(&resolved, g_static_scratch) != cudaSuccess || !resolved) return KVB_ERR_CUDA;
+    g_scratch_addr[device].store(resolved, std::memory_order_release);
   }
-  unsigned long long* base = static_cast<unsigned long long*>(g_scratch_addr[device]);
+  unsigned long long* base = static_cast<unsigned long long*>(resolved);
   ReqDesc* desc_dev = reinterpret_cast<ReqDesc*>(base);
   unsigned long long* acc = base + kDescWords;
 

@@ -4,6 +4,7 @@
 #include <stdarg.h>
 #include <stdio.h>
 #include <stdlib.h>
+#include <limits.h>
 #include <string.h>
 
 #include <new>
@@ -37,9 +38,10 @@ struct kvb_ctx {
   size_t arena_bytes = 0;
   bool acc_dirty = false;
   int n_sm = 0;
-  bool attn_legacy = false;  // KVB_ATTN=mma selects the warp-level mma.sync kernel (debug aid)
-  int attn_mode = 0;         // KVB_ATTN=onetile (2): one tile per CTA instead of persistent CTAs (cross-check)
-  bool force_copy = false;   // KVB_DESC=copy: descriptors always go by cudaMemcpyAsync (cross-check)
+  // debug options (kvb_set_debug_option); the defaults are the product path
+  bool attn_one_tile = false;  // one tile per attention CTA instead of persistent CTAs (cross-check)
+  bool force_copy = false;     // descriptors always go by cudaMemcpyAsync (cross-check)
+  bool pdl = true;             // programmatic dependent launch along the kernel chain
   cudaStream_t last_stream = nullptr;
   int64_t launches = 0;
   char err[512] = {0};
@@ -85,7 +87,7 @@ int take_slot(kvb_ctx* c, uint8_t** host) {
 int upload(kvb_ctx* c, int slot, const uint8_t* host, size_t bytes, cudaStream_t st, int rope_chunks = 0, bool* rope_done = nullptr) {
   if (rope_done) *rope_done = false;
   if (bytes <= kDescBlobBytes && !c->force_copy) {
-    KVB_CUDA(c, launch_store_blob(host, bytes, c->arena_dev, rope_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
+    KVB_CUDA(c, launch_store_blob(host, bytes, c->arena_dev, rope_chunks, c->inv_freq, c->model.d / 2, c->cs_table, c->pdl, st));
     c->slot_used[slot] = false;
     c->launches += 1;
     if (rope_done) *rope_done = rope_chunks > 0;
@@ -98,13 +100,14 @@ int upload(kvb_ctx* c, int slot, const uint8_t* host, size_t bytes, cudaStream_t
 }
 
 // Checks one request's table: chunks in prompt order tiling [0, T) exactly, enums and pointers sane.
-int check_request(kvb_ctx* c, const kvb_request& r, int ri, bool need_payload) {
+// need_fresh: the call reads the request's fresh tensor (the attention and the importance score do not).
+int check_request(kvb_ctx* c, const kvb_request& r, int ri, bool need_payload, bool need_fresh) {
   const int C = c->model.chunk_tokens;
   if (r.T <= 0 || r.n_chunks <= 0 || !r.chunks) return fail(c, KVB_ERR_INVALID_ARG, "request %d: empty or NULL chunk table", ri);
   if (r.T % C != 0 || r.n_chunks != r.T / C)
     return fail(c, KVB_ERR_BAD_TABLE, "request %d: T=%d is not n_chunks=%d x chunk_tokens=%d", ri, r.T, r.n_chunks, C);
-  if (!r.kv_buf || !r.fresh) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL kv_buf or fresh", ri);
-  if (!aligned16(r.kv_buf) || !aligned16(r.fresh))
+  if (!r.kv_buf || (need_fresh && !r.fresh)) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL kv_buf or fresh", ri);
+  if (!aligned16(r.kv_buf) || (need_fresh && !aligned16(r.fresh)))
     return fail(c, KVB_ERR_BAD_TABLE, "request %d: kv_buf / fresh must be 16-byte aligned", ri);
   for (int i = 0; i < r.n_chunks; ++i) {
     const kvb_chunk& k = r.chunks[i];
@@ -130,14 +133,15 @@ int check_request(kvb_ctx* c, const kvb_request& r, int ri, bool need_payload) {
   return KVB_OK;
 }
 
-int check_batch(kvb_ctx* c, const kvb_request* reqs, int n_req, bool need_payload, int* chunks_total, int64_t* tokens_total) {
+int check_batch(kvb_ctx* c, const kvb_request* reqs, int n_req, bool need_payload, int* chunks_total, int64_t* tokens_total,
+                bool need_fresh = true) {
   if (!c) return KVB_ERR_INVALID_ARG;
   if (n_req < 0 || (n_req > 0 && !reqs)) return fail(c, KVB_ERR_INVALID_ARG, "bad request array");
   if (n_req > c->limits.max_requests) return fail(c, KVB_ERR_WORKSPACE, "%d requests > max_requests=%d", n_req, c->limits.max_requests);
   int ch = 0;
   int64_t tk = 0;
   for (int r = 0; r < n_req; ++r) {
-    const int st = check_request(c, reqs[r], r, need_payload);
+    const int st = check_request(c, reqs[r], r, need_payload, need_fresh);
     if (st != KVB_OK) return st;
     ch += reqs[r].n_chunks;
     tk += reqs[r].T;
@@ -212,6 +216,10 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   const bool pow2_h = (m.Hkv & (m.Hkv - 1)) == 0 && m.Hkv <= 16;
   const bool pow2_rep = (rep & (rep - 1)) == 0 && rep <= 16;
   if (m.d != 128 || m.chunk_tokens != 128 || m.int4_group != 32 || !pow2_h || !pow2_rep) return KVB_ERR_UNSUPPORTED;
+  // the kernels index tokens, tiles and grid dimensions with 32 bits: a batch stays below 2^31 tokens
+  // (and chunk-layers), L below the grid's y limit
+  if (m.L > 65535 || limits->max_tokens_total > (int64_t)INT32_MAX || (int64_t)limits->max_chunks_total * m.L * 2 * m.Hkv > (int64_t)INT32_MAX)
+    return KVB_ERR_UNSUPPORTED;
 
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return KVB_ERR_NO_DEVICE;
@@ -236,15 +244,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   if (smem_max > 200 * 1024) return fail(c, KVB_ERR_UNSUPPORTED, "chunk-layer block of %zu bytes does not fit shared memory", smem_max);
   KVB_CUDA(c, assemble_configure(smem_max));
   KVB_CUDA(c, topk_configure());
-  KVB_CUDA(c, attention_mma_configure());
   KVB_CUDA(c, attention_tc_configure());
-  const char* attn_env = getenv("KVB_ATTN");
-  c->attn_legacy = attn_env && strcmp(attn_env, "mma") == 0;
-  const char* pdl_env = getenv("KVB_PDL");
-  pdl_enabled() = !(pdl_env && strcmp(pdl_env, "0") == 0);
-  const char* desc_env = getenv("KVB_DESC");
-  c->force_copy = desc_env && strcmp(desc_env, "copy") == 0;
-  c->attn_mode = attn_env && strcmp(attn_env, "persistent") == 0 ? 1 : (attn_env && strcmp(attn_env, "onetile") == 0 ? 2 : 0);
 
   const int half = m.d / 2;
   std::vector<double> inv(half);
@@ -264,6 +264,16 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, cudaMalloc(&c->status_dev, sizeof(uint32_t)));
   KVB_CUDA(c, cudaMemset(c->status_dev, 0, sizeof(uint32_t)));
   KVB_CUDA(c, cudaDeviceSynchronize());
+  return KVB_OK;
+}
+
+int kvb_set_debug_option(kvb_ctx* c, const char* key, int value) {
+  if (!c || !key) return KVB_ERR_INVALID_ARG;
+  if (value != 0 && value != 1) return fail(c, KVB_ERR_INVALID_ARG, "debug option values are 0 or 1");
+  if (strcmp(key, "dependent_launch") == 0) c->pdl = value != 0;
+  else if (strcmp(key, "descriptor_copy") == 0) c->force_copy = value != 0;
+  else if (strcmp(key, "attention_one_tile_per_cta") == 0) c->attn_one_tile = value != 0;
+  else return fail(c, KVB_ERR_INVALID_ARG, "unknown debug option '%s'", key);
   return KVB_OK;
 }
 
@@ -446,7 +456,7 @@ int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stre
     KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
     c->launches += 1;
   }
-  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, 0, nullptr, st));
+  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, 0, nullptr, c->pdl, st));
   c->launches += 1;
   return KVB_OK;
 }
@@ -482,7 +492,7 @@ int kvb_deviation_topk(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
   c->acc_dirty = true;  // cleared again once both kernels are in the stream
   KVB_CUDA(c, launch_deviation(rd_dev, n_req, ext.tiles, c->dims, p->which, c->acc, st));
   KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_deviation_terms(c, p->which), ext.max_T, ext.max_k, c->acc,
-                          c->status_dev, st));
+                          c->status_dev, c->pdl, st));
   c->acc_dirty = false;
   c->launches += 2;
   return KVB_OK;
@@ -526,9 +536,9 @@ int kvb_assemble_select(kvb_ctx* c, const kvb_request* reqs, int n_req, const kv
     c->launches += 1;
   }
   c->acc_dirty = true;  // cleared again once both kernels are in the stream
-  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, p->which, c->acc, st));
+  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, p->which, c->acc, c->pdl, st));
   KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_deviation_terms(c, p->which), ext.max_T, ext.max_k, c->acc,
-                          c->status_dev, st));
+                          c->status_dev, c->pdl, st));
   c->acc_dirty = false;
   c->launches += 2;
   return KVB_OK;
@@ -538,7 +548,7 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
                        void* const* out, float softmax_scale, void* cuda_stream) {
   int n_chunks = 0;
   int64_t n_tok = 0;
-  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
+  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok, false);
   if (st0 != KVB_OK) return st0;
   if (n_req == 0) return KVB_OK;
   if (!sel || !q || !out) return fail(c, KVB_ERR_INVALID_ARG, "NULL selection, q or out array");
@@ -579,10 +589,8 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
     }
     rd[r] = d;
     tiles += (s.sel_capacity + tok_per_tile - 1) / tok_per_tile;
-    if (!c->attn_legacy) {
-      const int e = attention_tc_encode_maps(c->dims, q[r], s.sel_capacity, reqs[r].kv_buf, reqs[r].T, host + maps_off + 256 * (size_t)r);
-      if (e != 0) return fail(c, KVB_ERR_CUDA, "request %d: tensor map encoding failed (%d)", r, e);
-    }
+    const int e = attention_tc_encode_maps(c->dims, q[r], s.sel_capacity, reqs[r].kv_buf, reqs[r].T, host + maps_off + 256 * (size_t)r);
+    if (e != 0) return fail(c, KVB_ERR_CUDA, "request %d: tensor map encoding failed (%d)", r, e);
   }
   const size_t counter_off = maps_off + 256 * (size_t)n_req;  // the attention kernel's tile counter, uploaded as zero
   memset(host + counter_off, 0, 128);
@@ -591,13 +599,9 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
   c->last_stream = st;
   const ReqDesc* rd_dev = reinterpret_cast<const ReqDesc*>(c->arena_dev);
   // persistent CTAs measured faster at every prompt length (most for short prompts, whose tiles are a
-  // few sub-blocks long); KVB_ATTN=onetile selects one tile per CTA (cross-check)
-  const bool persistent = c->attn_mode != 2;
-  if (c->attn_legacy)
-    KVB_CUDA(c, launch_attention_mma(rd_dev, n_req, tiles, c->dims, softmax_scale, st));
-  else
-    KVB_CUDA(c, launch_attention_tc(rd_dev, c->arena_dev + maps_off, n_req, tiles, c->dims, softmax_scale, c->status_dev,
-                                    reinterpret_cast<unsigned int*>(c->arena_dev + counter_off), c->n_sm, persistent, st));
+  // few sub-blocks long); the debug option selects one tile per CTA (cross-check)
+  KVB_CUDA(c, launch_attention_tc(rd_dev, c->arena_dev + maps_off, n_req, tiles, c->dims, softmax_scale, c->status_dev,
+                                  reinterpret_cast<unsigned int*>(c->arena_dev + counter_off), c->n_sm, !c->attn_one_tile, c->pdl, st));
   c->launches += 1;
   return KVB_OK;
 }
@@ -643,7 +647,7 @@ int kvb_patch(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_selectio
 int kvb_chunk_importance(kvb_ctx* c, const kvb_request* reqs, int n_req, float* const* importance, void* cuda_stream) {
   int n_chunks = 0;
   int64_t n_tok = 0;
-  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok);
+  const int st0 = check_batch(c, reqs, n_req, false, &n_chunks, &n_tok, false);
   if (st0 != KVB_OK) return st0;
   if (n_req == 0) return KVB_OK;
   if (!importance) return fail(c, KVB_ERR_INVALID_ARG, "NULL importance array");

@@ -60,6 +60,7 @@ struct ModelDims {
 };
 
 // ---- launchers (each defined next to its kernel) ----
+// pdl: launch with the programmatic-dependent-launch attribute (csrc/pdl.cuh); a context option.
 // Tables of at most kDescBlobBytes go to the arena as a kernel argument (csrc/desc_store.cu; two
 // argument sizes, 3840 and 16384 bytes, so a small call does not pay for a large argument); the
 // chunk descriptors, if any, must be at the start of the bytes, and n_rope_chunks > 0 also fills
@@ -67,12 +68,12 @@ struct ModelDims {
 constexpr size_t kDescBlobSmall = 3840;
 constexpr size_t kDescBlobBytes = 16384;
 cudaError_t launch_store_blob(const void* host_bytes, size_t bytes, uint8_t* dst, int n_rope_chunks, const double* inv_freq,
-                              int half_d, float2* cs_table, cudaStream_t st);
+                              int half_d, float2* cs_table, bool pdl, cudaStream_t st);
 // launch_assemble: acc != NULL fuses the deviation sums (which: bit 0 keys, bit 1 values) into the stitch.
 cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const double* inv_freq, int half_d,
                               float2* cs_table, cudaStream_t st);
 cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
-                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, cudaStream_t st);
+                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, bool pdl, cudaStream_t st);
 size_t assemble_smem_bytes(const ModelDims& m, int mode);
 cudaError_t assemble_configure(size_t max_smem);
 
@@ -81,14 +82,10 @@ cudaError_t launch_deviation(const ReqDesc* reqs, int n_req, int total_tiles, co
 int deviation_tile_tokens();
 
 cudaError_t launch_topk(const ReqDesc* reqs, int n_req, const SeamWindow* seams, const ModelDims& m, int n_terms,
-                        int max_T, int max_k, unsigned long long* acc, uint32_t* status, cudaStream_t st);
+                        int max_T, int max_k, unsigned long long* acc, uint32_t* status, bool pdl, cudaStream_t st);
 cudaError_t topk_configure();
 int topk_max_T();
 int topk_max_k();
-
-cudaError_t launch_attention_mma(const ReqDesc* reqs, int n_req, int total_tiles, const ModelDims& m, float scale,
-                                 cudaStream_t st);
-cudaError_t attention_mma_configure();
 
 cudaError_t attention_tc_configure();
 // One warp waits on a barrier nothing completes; gives up after limit_ns and raises DEV_STATUS_WAIT_TIMEOUT.
@@ -99,7 +96,7 @@ int attention_tc_encode_maps(const ModelDims& m, const void* q, int sel_capacity
 // n_sm: SMs of the device
 cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req, int total_tiles, const ModelDims& m,
                                 float scale, uint32_t* status, unsigned int* tile_counter, int n_sm, bool persistent,
-                                cudaStream_t st);
+                                bool pdl, cudaStream_t st);
 
 cudaError_t launch_patch(const ReqDesc* reqs, int n_req, int total_tiles, int rows_per_cta, const ModelDims& m,
                          cudaStream_t st);

@@ -341,13 +341,13 @@ cudaError_t topk_configure() {
 }
 
 cudaError_t launch_topk(const ReqDesc* reqs, int n_req, const SeamWindow* seams, const ModelDims& m, int n_terms,
-                        int max_T, int max_k, unsigned long long* acc, uint32_t* status, cudaStream_t st) {
+                        int max_T, int max_k, unsigned long long* acc, uint32_t* status, bool pdl, cudaStream_t st) {
   (void)m;
   int t_pad = (max_T + 31) & ~31;
   int k_pad = 1;
   while (k_pad < max_k) k_pad <<= 1;
   const float inv_scale = (float)(1.0 / (1099511627776.0 * (double)n_terms));  // 2^-40 / n_terms
-  return launch_pdl(topk_kernel, dim3(n_req), dim3(kThreads), topk_smem(t_pad, k_pad), st, reqs, seams, inv_scale, acc, t_pad, status);
+  return launch_pdl(pdl, topk_kernel, dim3(n_req), dim3(kThreads), topk_smem(t_pad, k_pad), st, reqs, seams, inv_scale, acc, t_pad, status);
 }
 
 }  // namespace kvb

@@ -11,7 +11,7 @@ from paper_2608_21362_b200 import binding as B
 from paper_2608_21362_b200 import synth
 from paper_2608_21362_b200.build import build_library
 
-import helpers
+import oracle_glue as helpers
 from test_gpu_parity import check_assembled, check_attention, check_selection, oracle_stitch, prepare, run_assemble, run_attention, run_select
 
 pytestmark = pytest.mark.gpu
@@ -122,21 +122,24 @@ def test_attention_sink_tokens_join_the_selection():
         B.kvb_destroy(ctx)
 
 
-def test_descriptor_upload_paths_agree(monkeypatch):
+def test_descriptor_upload_paths_agree():
     """Small calls send their tables as a kernel argument (and fill the rotation table in the same
-    launch); KVB_DESC=copy forces the pinned-buffer copy and the separate table kernel.  Same bits."""
+    launch); the context's "descriptor_copy" option forces the pinned-buffer copy and the separate table
+    kernel, "dependent_launch" = 0 launches the chain without programmatic dependent launch.  Same bits."""
     wl = synth.workload(0)
     sh = wl.shape
     got = {}
-    for mode in ("kernel", "copy"):
-        if mode == "copy":
-            monkeypatch.setenv("KVB_DESC", "copy")
-        else:
-            monkeypatch.delenv("KVB_DESC", raising=False)
+    for mode in ("kernel", "copy", "no_pdl"):
         reqs = prepare(wl)
         (r,) = reqs
         ctx = B.create_for_shape(sh, 0)
         try:
+            if mode == "copy":
+                B.kvb_set_debug_option(ctx, "descriptor_copy", 1)
+            if mode == "no_pdl":
+                B.kvb_set_debug_option(ctx, "dependent_launch", 0)
+            assert B.kvb_set_debug_option(ctx, "no_such_option", 1, check=False) == B.KVB_ERR_INVALID_ARG
+            assert B.kvb_set_debug_option(ctx, "descriptor_copy", 2, check=False) == B.KVB_ERR_INVALID_ARG
             before = B.kvb_launch_count(ctx)
             tbl = B.RequestTable(reqs)
             k = B.kvb_select_count(r.plan.T, 0.15)
@@ -146,12 +149,13 @@ def test_descriptor_upload_paths_agree(monkeypatch):
             B.kvb_selective_attn(ctx, tbl, sel, [r.q], [out], 0.1)
             B.kvb_last_status(ctx)
             # kernel path: store+table, stitch, selection; store, attention.  copy path: table, stitch, selection; attention
-            assert B.kvb_launch_count(ctx) - before == (5 if mode == "kernel" else 4)
+            assert B.kvb_launch_count(ctx) - before == (4 if mode == "copy" else 5)
             got[mode] = (r.kv_buf.view(torch.int16).clone(), sel.delta[0].clone(), sel.sel[0].clone(), out.view(torch.int16).clone())
         finally:
             B.kvb_destroy(ctx)
-    for a, b in zip(got["kernel"], got["copy"]):
-        assert torch.equal(a, b)
+    for other in ("copy", "no_pdl"):
+        for a, b in zip(got["kernel"], got[other]):
+            assert torch.equal(a, b)
 
 
 def test_selection_overflow_is_reported_once_and_cut_cleanly():
@@ -186,9 +190,9 @@ def test_selection_overflow_is_reported_once_and_cut_cleanly():
         B.kvb_destroy(ctx)
 
 
-def test_attention_persistent_and_one_tile_ctas_agree(monkeypatch):
-    """The attention kernel runs either as persistent CTAs drawing tiles from a counter (short prompts)
-    or with one tile per CTA (long prompts); KVB_ATTN forces either.  Both must give the same bits, on
+def test_attention_persistent_and_one_tile_ctas_agree():
+    """The attention kernel runs as persistent CTAs drawing tiles from a counter; the context's
+    "attention_one_tile_per_cta" option runs one tile per CTA instead.  Both must give the same bits, on
     a batch whose tiles are short, ragged and partly empty (sel_capacity = T > n_sel)."""
     sh = synth.Shape(L=3, Hq=16, Hkv=2)
     plans = [synth._request(T, sh.C, [synth.MODE_INT8] * (T // sh.C), [((5 * i) % (T // sh.C)) * sh.C for i in range(T // sh.C)]) for T in (128, 640, 1152, 256)]
@@ -196,9 +200,9 @@ def test_attention_persistent_and_one_tile_ctas_agree(monkeypatch):
     reqs = prepare(wl)
     outs = {}
     for mode in ("persistent", "onetile"):
-        monkeypatch.setenv("KVB_ATTN", mode)
         ctx = B.create_for_shape(sh, 0, max_requests=len(reqs))
         try:
+            B.kvb_set_debug_option(ctx, "attention_one_tile_per_cta", int(mode == "onetile"))
             tbl = run_assemble(ctx, reqs)
             Ts = [r.plan.T for r in reqs]
             ks = [B.kvb_select_count(T, 0.2) for T in Ts]

@@ -18,7 +18,7 @@ from paper_2608_21362_b200 import synth
 from paper_2608_21362_b200.build import build_library
 
 import bench
-import helpers
+import oracle_glue as helpers
 from test_gpu_parity import ulp16
 
 pytestmark = pytest.mark.gpu

@@ -8,7 +8,7 @@ from paper_2608_21362_b200 import binding as B
 from paper_2608_21362_b200 import synth
 from paper_2608_21362_b200.build import build_library
 
-import helpers
+import oracle_glue as helpers
 from test_gpu_parity import _mixed_workload, check_assembled, check_selection, oracle_stitch, prepare, run_assemble, run_select
 
 pytestmark = pytest.mark.gpu

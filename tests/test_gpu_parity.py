@@ -20,7 +20,7 @@ from paper_2608_21362_b200 import binding as B
 from paper_2608_21362_b200 import synth
 from paper_2608_21362_b200.build import build_library
 
-import helpers
+import oracle_glue as helpers
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -49,43 +49,7 @@ def to_device(reqs):
     return reqs
 
 
-def ulp16(y, kv_dtype):
-    a = np.abs(y)
-    e = np.floor(np.log2(np.maximum(a, 1e-300)))
-    if kv_dtype == "bf16":
-        return np.exp2(np.maximum(e, -126) - 7)
-    return np.exp2(np.maximum(e, -14) - 10)
-
-
-def check_assembled(sh, req, kv_gpu_bits, exact, kv_oracle_bits):
-    """Element-wise tolerance check of a stitched buffer plus a bit-agreement count."""
-    dtc = helpers.dt_code(sh)
-    g = oracle.bits_to_f64(kv_gpu_bits, dtc)
-    half = sh.d // 2
-    for ck in req.chunks:
-        sl = slice(ck.plan.new_pos, ck.plan.new_pos + sh.C)
-        if ck.plan.mode == synth.MODE_FRESH:
-            assert np.array_equal(kv_gpu_bits[:, :, sl], kv_oracle_bits[:, :, sl]), "fresh rows must be bit copies"
-            continue
-        y = exact[:, :, sl]  # [L,2,C,H,d]
-        M = np.abs(y).max(axis=(2, 3, 4), keepdims=True)
-        ref = np.abs(y).copy()
-        pair = np.sqrt(y[:, 0, ..., :half] ** 2 + y[:, 0, ..., half:] ** 2)
-        ref[:, 0, ..., :half] = pair
-        ref[:, 0, ..., half:] = pair
-        bound = 1e-3 * ref + 0.5 * ulp16(y, sh.kv_dtype) + 2e-6 * M
-        err = np.abs(g[:, :, sl] - y)
-        worst = float((err / bound).max())
-        assert worst <= 1.0, "chunk at %d (mode %d): error %.3g x bound" % (ck.plan.new_pos, ck.plan.mode, worst)
-    # Beyond the tolerance: how often the two 16-bit roundings coincide.  The GPU rounds a float32 result
-    # whose error e is a few 2^-24 of the chunk's magnitude M, the oracle rounds the exact value; they
-    # differ when y lies within e of a rounding boundary, i.e. with probability ~ 2e / ulp16(y)
-    # = c * 2^-23 * (M/|y|) / 2^-p (p = 8 bits for bf16, 11 for fp16; c ~ 2..3, mean M/|y| ~ 3):
-    # about 3e-4 in bf16 and 2e-3 in fp16 (measured: up to 2.2e-3 on int4 keys in fp16).
-    agree = float(np.mean(kv_gpu_bits == kv_oracle_bits))
-    floor = 0.999 if sh.kv_dtype == "bf16" else 0.995
-    assert agree > floor, "only %.5f of stored values equal the oracle's rounding bit for bit" % agree
-    return agree
+ulp16, check_assembled = helpers.ulp16, helpers.check_assembled
 
 
 def oracle_stitch(sh, req):

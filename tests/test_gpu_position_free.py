@@ -9,7 +9,7 @@ from paper_2608_21362_b200 import binding as B
 from paper_2608_21362_b200 import synth
 from paper_2608_21362_b200.build import build_library
 
-import helpers
+import oracle_glue as helpers
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"

@@ -4,7 +4,7 @@ import numpy as np
 import oracle
 from paper_2608_21362_b200 import synth
 
-import helpers
+import oracle_glue as helpers
 
 
 def test_cfg0_recipe_and_selection_finds_the_seams():
