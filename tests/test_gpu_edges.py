@@ -319,3 +319,55 @@ def test_a_barrier_wait_that_cannot_complete_gives_up_and_is_reported():
         check_attention(sh, r, sel.sel[0].cpu().numpy()[:n], out, None, None)
     finally:
         B.kvb_destroy(ctx)
+
+
+def test_selection_cluster_path_plateaus_windows_and_extremes():
+    """Prompts beyond 2048 positions are selected by a thread-block cluster, every CTA owning a slice:
+    thresholds that fall on plateaus of equal deviations spanning slice boundaries (taken lowest index
+    first), k = 0 / 1 / T - 1 / T, windows that straddle slices, a slice count that does not divide the
+    prompt, and a batch that mixes short and long prompts.  rank / sel / n_sel must equal the oracle's
+    selection of the GPU's own delta, bit for bit."""
+    sh = synth.Shape(L=2, Hq=16, Hkv=2)
+    Ts = (4224, 16384, 640, 8192 + 128)  # 3, 8, (8), 5 slices of unequal fill; the short prompt shares the launch
+    rng = np.random.default_rng(11)
+
+    class R:
+        pass
+
+    reqs = []
+    for T in Ts:
+        r = R()
+        modes = [synth.MODE_FP16 if (i % 5) else synth.MODE_FRESH for i in range(T // sh.C)]
+        r.plan = synth._request(T, sh.C, modes, [i * sh.C for i in range(T // sh.C)])
+        r.chunks = [synth.Chunk(cp) for cp in r.plan.chunks]
+        g = torch.Generator(device=DEV).manual_seed(T)
+        r.kv_buf = torch.randn((sh.L, 2, T, sh.Hkv, sh.d), generator=g, device=DEV).to(torch.bfloat16)
+        noise = 0.02 * torch.randn(r.kv_buf.shape, generator=g, device=DEV)
+        r.fresh = (r.kv_buf.float() + noise).to(torch.bfloat16)
+        # plateaus: long runs of exact copies (delta 0), and groups of positions that repeat one (stored, fresh) pair
+        r.fresh[:, :, T // 3 : T // 3 + T // 4] = r.kv_buf[:, :, T // 3 : T // 3 + T // 4]
+        src = int(rng.integers(0, T // 3))
+        for dst in rng.choice(np.arange(T // 3 + T // 4, T), size=T // 16, replace=False):
+            r.kv_buf[:, :, dst] = r.kv_buf[:, :, src]
+            r.fresh[:, :, dst] = r.fresh[:, :, src]
+        reqs.append(r)
+    ctx = B.create_for_shape(sh, 0, max_requests=len(reqs), max_chunks_total=sum(T // sh.C for T in Ts), max_tokens_total=sum(Ts))
+    try:
+        # the whole batch (k up to the kernel's limit of 8192), then the 4224-token prompt alone with k = T - 1 and k = T
+        cases = [(reqs, Ts, c) for c in ((0.15, -1, 16, 0, 0), (0.45, -1, 40, 40, 100), (0.0, 0, 0, 0, 0), (0.0, 1, 0, 0, 0), (0.5, -1, 0, 0, 4000))]
+        cases += [(reqs[:1], Ts[:1], c) for c in ((1.0, -1, 0, 0, 0), (0.9999, -1, 3, 3, 0))]
+        for rs, ts, (ratio, k_over, before, after, sinks) in cases:
+            tbl = B.RequestTable(rs)
+            ks = [k_over if k_over >= 0 else B.kvb_select_count(T, ratio) for T in ts]
+            sel = B.SelectionTable(ts, ks, ts, DEV)
+            B.kvb_deviation_topk(ctx, tbl, ratio, k_over, before, after, 3, sel, sink_tokens=sinks)
+            B.kvb_last_status(ctx)
+            for i, (r, T, k) in enumerate(zip(rs, ts, ks)):
+                dg = sel.delta[i].cpu().numpy()
+                want_rank = oracle.topk(dg, k)
+                assert np.array_equal(sel.rank[i].cpu().numpy()[:k], want_rank), (T, k)
+                want = oracle.seam_select(want_rank, [c.plan.new_pos for c in r.chunks], [c.plan.mode for c in r.chunks], T, before, after, sinks)
+                n = int(sel.n_sel[i])
+                assert n == len(want) and np.array_equal(sel.sel[i].cpu().numpy()[:n], want), (T, k)
+    finally:
+        B.kvb_destroy(ctx)
