@@ -98,6 +98,10 @@ typedef struct {
   const kvb_chunk* chunks; /* host */
   void* kv_buf;            /* device, [L][2][T][H][d], written by kvb_assemble */
   const void* fresh;       /* device, same shape and dtype: freshly projected K~, V~ of every position */
+  float* importance;       /* device, optional (NULL: not wanted): [n_chunks] float32.  kvb_assemble and
+                              kvb_assemble_select write every chunk's importance score (KV Cache Manager,
+                              Eq. 7: mean L2 norm of the chunk's stitched keys over layers, KV heads and
+                              tokens) from the key rows they hold while stitching; other calls ignore it */
 } kvb_request;
 
 typedef struct {
@@ -197,7 +201,9 @@ int kvb_patch(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_select
  * tokens of chunk c of ||k||_2, read from the stitched kv_buf (a rotation
  * leaves the norms unchanged).  importance: host array of n_req device
  * pointers, each to n_chunks float32 values.  reqs[r].fresh is not read and
- * may be NULL. */
+ * may be NULL.  For callers that only hold a stitched buffer: a stitching call
+ * delivers the same scores without this second read of the keys when
+ * kvb_request.importance is set. */
 int kvb_chunk_importance(kvb_ctx* ctx, const kvb_request* reqs, int n_req, float* const* importance,
                          void* cuda_stream);
 

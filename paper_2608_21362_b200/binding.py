@@ -47,6 +47,7 @@ class kvb_request(C.Structure):
         ("chunks", C.POINTER(kvb_chunk)),
         ("kv_buf", C.c_void_p),
         ("fresh", C.c_void_p),
+        ("importance", C.c_void_p),
     ]
 
 
@@ -121,7 +122,7 @@ class RequestTable:
 
     def __init__(self, requests: Sequence, chunk_tokens: int = 128):
         """requests: objects with .plan.T, .chunks (each .plan.{orig_pos,new_pos,mode,match} and the
-        four tensors or None), .kv_buf, .fresh -- e.g. synth.Request."""
+        four tensors or None), .kv_buf, .fresh, optionally .importance -- e.g. synth.Request."""
         self._keep = []
         n = len(requests)
         self.n = n
@@ -146,6 +147,10 @@ class RequestTable:
             self.array[r].kv_buf = rq.kv_buf.data_ptr()
             self.array[r].fresh = rq.fresh.data_ptr()
             self._keep += [rq.kv_buf, rq.fresh]
+            imp = getattr(rq, "importance", None)  # optional [n_chunks] float32 tensor: Eq. 7 from the stitch
+            if imp is not None:
+                self.array[r].importance = imp.data_ptr()
+                self._keep.append(imp)
 
 
 class SelectionTable:

@@ -127,12 +127,13 @@ __device__ __forceinline__ void copy_rows(uint8_t* dst, const uint8_t* src, size
   for (; i < n; i += kThreads) d[i] = __ldcs(s + i);
 }
 
-// Copy of `rows` 256-byte (token, head) rows (a multiple of 32) that also accumulates each row's
-// deviation term against the fresh tensor: a half-warp per row, two rows per pass.
-// acc_tok points at the accumulator of the first row's token.
+// Copy of `rows` 256-byte (token, head) rows (a multiple of 32) that also takes each row's sums: a
+// half-warp per row, two rows per pass.  dev_on: the row's deviation term against the fresh tensor
+// goes to the accumulator of its token (acc_tok points at the first row's token).  norm_on: the
+// row's L2 norm is added to norm_part on lanes 0 and 8 of the half-warp (Eq. 7).
 template <int DT>
 __device__ __forceinline__ void copy_rows_dev(uint8_t* dst, const uint8_t* src, const uint8_t* fresh, int rows, int H,
-                                              int tid, unsigned long long* acc_tok) {
+                                              int tid, unsigned long long* acc_tok, bool dev_on, bool norm_on, float& norm_part) {
   const int lane = tid & 31, s = lane >> 4, ln = lane & 15;
   const int hw = (tid >> 5) * 2 + s;
   const bool heads_paired = (H & 1) == 0;  // rows 2w, 2w+1 of a warp belong to one token
@@ -140,26 +141,49 @@ __device__ __forceinline__ void copy_rows_dev(uint8_t* dst, const uint8_t* src, 
     const int ub = ua + 16;
     const size_t oa = (size_t)ua * 256 + (size_t)ln * 16, ob = (size_t)ub * 256 + (size_t)ln * 16;
     const uint4 a0 = __ldcs(reinterpret_cast<const uint4*>(src + oa)), a1 = __ldcs(reinterpret_cast<const uint4*>(src + ob));
-    const uint4 b0 = __ldcs(reinterpret_cast<const uint4*>(fresh + oa)), b1 = __ldcs(reinterpret_cast<const uint4*>(fresh + ob));
+    uint4 b0 = a0, b1 = a1;  // without the deviation only the norms are wanted
+    if (dev_on) b0 = __ldcs(reinterpret_cast<const uint4*>(fresh + oa)), b1 = __ldcs(reinterpret_cast<const uint4*>(fresh + ob));
     *reinterpret_cast<uint4*>(dst + oa) = a0;
     *reinterpret_cast<uint4*>(dst + ob) = a1;
-    float sa[3], sb[3];
+    float sa[3], sb[3], na2;
     row_sums<DT>(a0, b0, sa[0], sa[1], sa[2]);
     row_sums<DT>(a1, b1, sb[0], sb[1], sb[2]);
-    long long fx = pair_terms_fixed(sa, sb, ln, true, true);
-    if (heads_paired) fx += __shfl_xor_sync(0xffffffffu, fx, 16);
-    if ((ln & 7) == 0 && (!heads_paired || s == 0)) atomicAdd(acc_tok + ((ln & 8) ? ub : ua) / H, (unsigned long long)fx);
+    long long fx = pair_terms_fixed(sa, sb, ln, true, true, na2);
+    if (norm_on && (ln & 7) == 0) norm_part += sqrt_fast(na2);
+    if (dev_on) {
+      if (heads_paired) fx += __shfl_xor_sync(0xffffffffu, fx, 16);
+      if ((ln & 7) == 0 && (!heads_paired || s == 0)) atomicAdd(acc_tok + ((ln & 8) ? ub : ua) / H, (unsigned long long)fx);
+    }
   }
 }
 
-// DEV = true adds the deviation of every written row against the fresh tensor (Algorithm 2, step 2)
-// to acc[token]: K rows when which & 1, V rows when which & 2.
-template <typename OutT, bool DEV>
+// Sum of the CTA's norm parts (held by lanes 0 and 8 of every half-warp), added up in a fixed order
+// and written as one double: the chunk-layer's share of the importance score.
+__device__ __forceinline__ void store_norm_sum(float part, int tid, float* s_part, double* out) {
+  part += __shfl_xor_sync(0xffffffffu, part, 8);
+  part += __shfl_xor_sync(0xffffffffu, part, 16);
+  if ((tid & 31) == 0) s_part[tid >> 5] = part;
+  __syncthreads();
+  if (tid == 0) {
+    double tot = 0.0;
+    for (int w = 0; w < kThreads / 32; ++w) tot += (double)s_part[w];
+    *out = tot;
+  }
+}
+
+// DEV = true takes the sums of every written row while it is in registers: its deviation against the
+// fresh tensor (Algorithm 2, step 2) goes to acc[token] -- K rows when which & 1, V rows when
+// which & 2.  NORM = true (a variant of DEV = true) also adds up the L2 norms of the key rows of this
+// chunk-layer into norm_sums[chunk][layer][part]: the importance score, Eq. 7, as a by-product of
+// the stitch.
+template <typename OutT, bool DEV, bool NORM>
 __global__ void __launch_bounds__(kThreads, 3)
     assemble_kernel(const ChunkDesc* __restrict__ chunks, const float2* __restrict__ cs_table, ModelDims m,
-                    uint32_t* __restrict__ status, int which, unsigned long long* __restrict__ acc) {
+                    uint32_t* __restrict__ status, int which, unsigned long long* __restrict__ acc,
+                    double* __restrict__ norm_sums) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) uint64_t bars[kParts + 1];
+  __shared__ float s_norm[kThreads / 32];
 
   pdl_wait();  // the descriptors and the rotation table come from the kernel before this one
   const int tid = threadIdx.x;
@@ -181,20 +205,30 @@ __global__ void __launch_bounds__(kThreads, 3)
   const size_t out_bytes = (size_t)C * row_elems * 2;
   const size_t layer_out_bytes = (size_t)m.C * row_elems * 2;
 
-  const bool dev_on = DEV && (which & (kv ? 2 : 1));
-  unsigned long long* acc_tok = DEV ? acc + cd.tok_offset + cd.new_pos + tb : nullptr;  // this CTA's first token
+  const bool dev_on = DEV && acc != nullptr && (which & (kv ? 2 : 1));
+  const bool norm_on = NORM && kv == 0;
+  unsigned long long* acc_tok = dev_on ? acc + cd.tok_offset + cd.new_pos + tb : nullptr;  // this CTA's first token
+  auto norm_out = [&]() { return norm_sums + ((size_t)ci * m.L + l) * split + part_id; };  // this CTA's slot
+  float norm_part = 0.f;  // lanes 0 and 8 of each half-warp: norms of the rows they reduced
 
   // ---- rows that are plain copies: FRESH chunks (deviation 0); unquantised values; unquantised keys that do not move
   if (cd.mode == KVB_MODE_FRESH) {
-    copy_rows(reinterpret_cast<uint8_t*>(dst), cd.fresh + dst_off * 2, out_bytes, tid);
+    if (norm_on) {
+      copy_rows_dev<Pack<OutT>::DT>(reinterpret_cast<uint8_t*>(dst), cd.fresh + dst_off * 2, nullptr, C * H, H, tid, nullptr, false, true, norm_part);
+      store_norm_sum(norm_part, tid, s_norm, norm_out());
+    } else {
+      copy_rows(reinterpret_cast<uint8_t*>(dst), cd.fresh + dst_off * 2, out_bytes, tid);
+    }
     return;
   }
   if (cd.mode == KVB_MODE_FP16 && (kv == 1 || cd.delta_pos == 0)) {
     const uint8_t* src = (kv ? cd.v_src : cd.k_src) + (size_t)l * layer_out_bytes + (size_t)tb * row_elems * 2;
-    if (dev_on)
-      copy_rows_dev<Pack<OutT>::DT>(reinterpret_cast<uint8_t*>(dst), src, cd.fresh + dst_off * 2, C * H, H, tid, acc_tok);
-    else
+    if (dev_on || norm_on) {
+      copy_rows_dev<Pack<OutT>::DT>(reinterpret_cast<uint8_t*>(dst), src, cd.fresh + dst_off * 2, C * H, H, tid, acc_tok, dev_on, norm_on, norm_part);
+      if (norm_on) store_norm_sum(norm_part, tid, s_norm, norm_out());
+    } else {
       copy_rows(reinterpret_cast<uint8_t*>(dst), src, out_bytes, tid);
+    }
     return;
   }
 
@@ -289,7 +323,7 @@ __global__ void __launch_bounds__(kThreads, 3)
       ok = ok && mbar_wait(&bars[1 + part], 0);
       ready_part = part;
     }
-    if (DEV) ok = __all_sync(0xffffffffu, ok);  // the deviation's shuffles need the whole warp
+    if (DEV) ok = __all_sync(0xffffffffu, ok);  // the row sums' shuffles need the whole warp
     return ok;
   };
   // Deviation terms of tokens t and t+1 of this half-warp's head: the stored words are still in
@@ -304,15 +338,23 @@ __global__ void __launch_bounds__(kThreads, 3)
     f[2] = __ldcs(reinterpret_cast<const uint2*>(f1)), f[3] = __ldcs(reinterpret_cast<const uint2*>(f1 + 128));
   };
   auto dev_pair = [&](int t, const uint2& wl0, const uint2& wh0, const uint2& wl1, const uint2& wh1, const uint2 (&f)[4]) {
-    const uint32_t a0[4] = {wl0.x, wl0.y, wh0.x, wh0.y}, b0[4] = {f[0].x, f[0].y, f[1].x, f[1].y};
-    const uint32_t a1[4] = {wl1.x, wl1.y, wh1.x, wh1.y}, b1[4] = {f[2].x, f[2].y, f[3].x, f[3].y};
-    float sa[3], sb[3];
-    row_sums4<Pack<OutT>::DT>(a0, b0, sa[0], sa[1], sa[2]);
-    row_sums4<Pack<OutT>::DT>(a1, b1, sb[0], sb[1], sb[2]);
-    long long fx = pair_terms_fixed(sa, sb, ln, true, true);
-    const bool heads_paired = (H & 1) == 0;  // the warp's two half-warps hold two heads of the same tokens
-    if (heads_paired) fx += __shfl_xor_sync(0xffffffffu, fx, 16);
-    if ((ln & 7) == 0 && (!heads_paired || s == 0)) atomicAdd(acc_tok + t + (ln >> 3), (unsigned long long)fx);
+    const uint32_t a0[4] = {wl0.x, wl0.y, wh0.x, wh0.y}, a1[4] = {wl1.x, wl1.y, wh1.x, wh1.y};
+    float sa[3], sb[3], na2;
+    if (dev_on) {
+      const uint32_t b0[4] = {f[0].x, f[0].y, f[1].x, f[1].y}, b1[4] = {f[2].x, f[2].y, f[3].x, f[3].y};
+      row_sums4<Pack<OutT>::DT>(a0, b0, sa[0], sa[1], sa[2]);
+      row_sums4<Pack<OutT>::DT>(a1, b1, sb[0], sb[1], sb[2]);
+    } else {  // only the norms are wanted
+      row_sums4<Pack<OutT>::DT>(a0, a0, sa[0], sa[1], sa[2]);
+      row_sums4<Pack<OutT>::DT>(a1, a1, sb[0], sb[1], sb[2]);
+    }
+    long long fx = pair_terms_fixed(sa, sb, ln, true, true, na2);
+    if (norm_on && (ln & 7) == 0) norm_part += sqrt_fast(na2);
+    if (dev_on) {
+      const bool heads_paired = (H & 1) == 0;  // the warp's two half-warps hold two heads of the same tokens
+      if (heads_paired) fx += __shfl_xor_sync(0xffffffffu, fx, 16);
+      if ((ln & 7) == 0 && (!heads_paired || s == 0)) atomicAdd(acc_tok + t + (ln >> 3), (unsigned long long)fx);
+    }
   };
 
   if (!kv) {
@@ -405,7 +447,7 @@ __global__ void __launch_bounds__(kThreads, 3)
       uint2 wl0, wh0, wl1, wh1;
       key_row(t, wl0, wh0);
       key_row(t + 1, wl1, wh1);
-      if (dev_on) {
+      if (dev_on || norm_on) {
         dev_pair(t, wl0, wh0, wl1, wh1, fr);
 #pragma unroll
         for (int i = 0; i < 4; ++i) fr[i] = fr_next[i];
@@ -458,6 +500,7 @@ __global__ void __launch_bounds__(kThreads, 3)
     }
   }
 
+  if (norm_on) store_norm_sum(norm_part, tid, s_norm, norm_out());
   if (!ok) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
   // Every thread drains every barrier before the CTA may retire, so no bulk copy can still be
   // writing this CTA's shared memory when it is handed to the next CTA.
@@ -479,7 +522,30 @@ __global__ void rope_table_kernel(const ChunkDesc* __restrict__ chunks, int n_ch
   cs_table[i] = make_float2((float)c, (float)sn);
 }
 
+// Eq. 7 from the stitch's by-product: importance of chunk ci = sum of its chunk-layers' norm sums
+// (added in layer order) / (L * H * C).  One thread per chunk descriptor.
+__global__ void importance_finalize_kernel(const ChunkDesc* __restrict__ chunks, int n_chunks, int parts_per_chunk,
+                                           const double* __restrict__ norm_sums, double inv_rows) {
+  const int ci = blockIdx.x * blockDim.x + threadIdx.x;
+  if (ci >= n_chunks) return;
+  float* out = chunks[ci].imp_out;
+  if (!out) return;
+  double tot = 0.0;
+  for (int i = 0; i < parts_per_chunk; ++i) tot += norm_sums[(size_t)ci * parts_per_chunk + i];
+  *out = (float)(tot * inv_rows);
+}
+
 }  // namespace
+
+int assemble_parts_per_layer(int Hkv) { return assemble_split(Hkv); }
+
+cudaError_t launch_importance_finalize(const ChunkDesc* chunks, int n_chunks, const ModelDims& m, const double* norm_sums,
+                                       cudaStream_t st) {
+  const int parts = m.L * assemble_split(m.Hkv);
+  importance_finalize_kernel<<<(n_chunks + 127) / 128, 128, 0, st>>>(chunks, n_chunks, parts, norm_sums,
+                                                                    1.0 / ((double)m.L * m.Hkv * m.C));
+  return cudaGetLastError();
+}
 
 size_t assemble_smem_bytes(const ModelDims& m, int mode) {
   const size_t E = (size_t)m.Hkv * m.d;
@@ -498,8 +564,9 @@ size_t assemble_smem_bytes(const ModelDims& m, int mode) {
 }
 
 cudaError_t assemble_configure(size_t max_smem) {
-  const void* fns[4] = {(const void*)assemble_kernel<__nv_bfloat16, false>, (const void*)assemble_kernel<__nv_bfloat16, true>,
-                        (const void*)assemble_kernel<__half, false>, (const void*)assemble_kernel<__half, true>};
+  const void* fns[6] = {(const void*)assemble_kernel<__nv_bfloat16, false, false>, (const void*)assemble_kernel<__nv_bfloat16, true, false>,
+                        (const void*)assemble_kernel<__nv_bfloat16, true, true>,   (const void*)assemble_kernel<__half, false, false>,
+                        (const void*)assemble_kernel<__half, true, false>,         (const void*)assemble_kernel<__half, true, true>};
   for (const void* f : fns) {
     cudaError_t e = cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem);
     if (e != cudaSuccess) return e;
@@ -515,21 +582,20 @@ cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const doubl
 }
 
 cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
-                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, bool pdl, cudaStream_t st) {
+                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, double* norm_sums,
+                            bool pdl, cudaStream_t st) {
   const unsigned grid = (unsigned)n_chunks * m.L * 2 * assemble_split(m.Hkv);
   const bool dev = acc != nullptr && (which & 3);
+  if (!dev) which = 0, acc = nullptr;
+  const dim3 g(grid), b(kThreads);
   if (m.dtype == KVB_DT_BF16) {
-    if (dev)
-      return launch_pdl(pdl, assemble_kernel<__nv_bfloat16, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
-    else
-      return launch_pdl(pdl, assemble_kernel<__nv_bfloat16, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
-  } else {
-    if (dev)
-      return launch_pdl(pdl, assemble_kernel<__half, true>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, which, acc);
-    else
-      return launch_pdl(pdl, assemble_kernel<__half, false>, dim3(grid), dim3(kThreads), smem_bytes, st, chunks, cs_table, m, status, 0, (unsigned long long*)nullptr);
+    if (norm_sums) return launch_pdl(pdl, assemble_kernel<__nv_bfloat16, true, true>, g, b, smem_bytes, st, chunks, cs_table, m, status, which, acc, norm_sums);
+    if (dev) return launch_pdl(pdl, assemble_kernel<__nv_bfloat16, true, false>, g, b, smem_bytes, st, chunks, cs_table, m, status, which, acc, norm_sums);
+    return launch_pdl(pdl, assemble_kernel<__nv_bfloat16, false, false>, g, b, smem_bytes, st, chunks, cs_table, m, status, which, acc, norm_sums);
   }
-  return cudaGetLastError();
+  if (norm_sums) return launch_pdl(pdl, assemble_kernel<__half, true, true>, g, b, smem_bytes, st, chunks, cs_table, m, status, which, acc, norm_sums);
+  if (dev) return launch_pdl(pdl, assemble_kernel<__half, true, false>, g, b, smem_bytes, st, chunks, cs_table, m, status, which, acc, norm_sums);
+  return launch_pdl(pdl, assemble_kernel<__half, false, false>, g, b, smem_bytes, st, chunks, cs_table, m, status, which, acc, norm_sums);
 }
 
 }  // namespace kvb

@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(kThreads)
     // lanes 0-7 hold the key sums of row u, lanes 8-15 the value sums
     float term = one_minus_cos(r0, r1, r2);
     if ((up && !useV) || (!up && !useK) || !live) term = 0.f;
-    long long fx = __float2ll_rn(term * kFixScale);
+    long long fx = term_to_fixed(term);
     fx += __shfl_xor_sync(0xffffffffu, fx, 8);  // K + V of row u
     if (pair_same_token) {
       fx += __shfl_xor_sync(0xffffffffu, fx, 16);  // both heads of the token

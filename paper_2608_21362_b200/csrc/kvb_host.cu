@@ -29,6 +29,7 @@ struct kvb_ctx {
   float2* cs_table = nullptr;            // [max_chunks][d/2] cos/sin of the chunk's rotation
   uint8_t* arena_dev = nullptr;          // descriptors of the current call
   unsigned long long* acc = nullptr;     // [max_tokens] fixed-point deviation sums (kept zero between calls)
+  double* norm_sums = nullptr;           // [max_chunks][L][parts] key-norm sums of the stitch (importance by-product)
   uint32_t* status_dev = nullptr;
   // pinned staging ring
   uint8_t* staging = nullptr;
@@ -261,6 +262,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   for (int s = 0; s < kSlots; ++s) KVB_CUDA(c, cudaEventCreateWithFlags(&c->slot_done[s], cudaEventDisableTiming));
   KVB_CUDA(c, cudaMalloc(&c->acc, (size_t)limits->max_tokens_total * sizeof(unsigned long long)));
   KVB_CUDA(c, cudaMemset(c->acc, 0, (size_t)limits->max_tokens_total * sizeof(unsigned long long)));
+  KVB_CUDA(c, cudaMalloc(&c->norm_sums, (size_t)limits->max_chunks_total * m.L * assemble_parts_per_layer(m.Hkv) * sizeof(double)));
   KVB_CUDA(c, cudaMalloc(&c->status_dev, sizeof(uint32_t)));
   KVB_CUDA(c, cudaMemset(c->status_dev, 0, sizeof(uint32_t)));
   KVB_CUDA(c, cudaDeviceSynchronize());
@@ -285,6 +287,7 @@ int kvb_destroy(kvb_ctx* c) {
   cudaFree(c->cs_table);
   cudaFree(c->arena_dev);
   cudaFree(c->acc);
+  cudaFree(c->norm_sums);
   cudaFree(c->status_dev);
   if (c->staging) cudaFreeHost(c->staging);
   for (int s = 0; s < kSlots; ++s)
@@ -318,8 +321,9 @@ namespace {
 // the kernel's last wave is made of short CTAs (cfg1: -6 % on the call).  A large batch keeps the
 // request order: there the tail is nothing and copy CTAs running among the decoding ones balance the
 // load/store and issue pipes better (cfg4: +3 % when sorted).
-size_t pack_chunks(kvb_ctx* c, const kvb_request* reqs, int n_req, ChunkDesc* cd) {
+size_t pack_chunks(kvb_ctx* c, const kvb_request* reqs, int n_req, ChunkDesc* cd, bool* any_importance) {
   size_t smem = 0;
+  *any_importance = false;
   int n = 0;
   long long n_chunks = 0;
   for (int r = 0; r < n_req; ++r) n_chunks += reqs[r].n_chunks;
@@ -343,6 +347,8 @@ size_t pack_chunks(kvb_ctx* c, const kvb_request* reqs, int n_req, ChunkDesc* cd
         d.mode = k.mode;
         d.tok_offset = tok;
         d.meta16 = k.meta_fp16;
+        d.imp_out = reqs[r].importance ? reqs[r].importance + i : nullptr;
+        if (d.imp_out) *any_importance = true;
         cd[n++] = d;
         const size_t s = assemble_smem_bytes(c->dims, k.mode);
         if (s > smem) smem = s;
@@ -446,7 +452,8 @@ int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stre
   const int slot_code = take_slot(c, &host);
   if (slot_code >= 0) return slot_code;
   const int slot = -slot_code - 1;
-  const size_t smem = pack_chunks(c, reqs, n_req, reinterpret_cast<ChunkDesc*>(host));
+  bool want_importance = false;
+  const size_t smem = pack_chunks(c, reqs, n_req, reinterpret_cast<ChunkDesc*>(host), &want_importance);
   bool rope_done = false;
   const int up = upload(c, slot, host, sizeof(ChunkDesc) * (size_t)n_chunks, st, n_chunks, &rope_done);
   if (up != KVB_OK) return up;
@@ -456,8 +463,13 @@ int kvb_assemble(kvb_ctx* c, const kvb_request* reqs, int n_req, void* cuda_stre
     KVB_CUDA(c, launch_rope_table(cd_dev, n_chunks, c->inv_freq, c->model.d / 2, c->cs_table, st));
     c->launches += 1;
   }
-  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, 0, nullptr, c->pdl, st));
+  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, 0, nullptr,
+                              want_importance ? c->norm_sums : nullptr, c->pdl, st));
   c->launches += 1;
+  if (want_importance) {
+    KVB_CUDA(c, launch_importance_finalize(cd_dev, n_chunks, c->dims, c->norm_sums, st));
+    c->launches += 1;
+  }
   return KVB_OK;
 }
 
@@ -517,7 +529,8 @@ int kvb_assemble_select(kvb_ctx* c, const kvb_request* reqs, int n_req, const kv
   // arena: chunk descriptors, then (256-byte aligned) request descriptors and the window list
   const size_t rd_off = (sizeof(ChunkDesc) * (size_t)n_chunks + 255) & ~(size_t)255;
   const size_t sw_off = rd_off + sizeof(ReqDesc) * (size_t)n_req;
-  const size_t smem = pack_chunks(c, reqs, n_req, reinterpret_cast<ChunkDesc*>(host));
+  bool want_importance = false;
+  const size_t smem = pack_chunks(c, reqs, n_req, reinterpret_cast<ChunkDesc*>(host), &want_importance);
   SelectExtent ext;
   const int st2 = pack_selection(c, reqs, n_req, p, out, reinterpret_cast<ReqDesc*>(host + rd_off),
                                  reinterpret_cast<SeamWindow*>(host + sw_off), &ext);
@@ -536,11 +549,16 @@ int kvb_assemble_select(kvb_ctx* c, const kvb_request* reqs, int n_req, const kv
     c->launches += 1;
   }
   c->acc_dirty = true;  // cleared again once both kernels are in the stream
-  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, p->which, c->acc, c->pdl, st));
+  KVB_CUDA(c, launch_assemble(cd_dev, n_chunks, c->cs_table, c->dims, smem, c->status_dev, p->which, c->acc,
+                              want_importance ? c->norm_sums : nullptr, c->pdl, st));
   KVB_CUDA(c, launch_topk(rd_dev, n_req, sw_dev, c->dims, n_deviation_terms(c, p->which), ext.max_T, ext.max_k, c->acc,
                           c->status_dev, c->pdl, st));
   c->acc_dirty = false;
   c->launches += 2;
+  if (want_importance) {  // after the selection, so the dependent-launch chain stitch -> selection stays as it is
+    KVB_CUDA(c, launch_importance_finalize(cd_dev, n_chunks, c->dims, c->norm_sums, st));
+    c->launches += 1;
+  }
   return KVB_OK;
 }
 

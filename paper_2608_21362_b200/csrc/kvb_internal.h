@@ -29,6 +29,7 @@ struct ChunkDesc {
   int32_t mode;
   int32_t tok_offset;    // first token of the request in the call's flat token space
   int32_t meta16;        // (scale, min) pairs are binary16 instead of float32
+  float* imp_out;        // where this chunk's importance score goes (NULL: not wanted)
 };
 
 // One request, as the deviation / top-k / attention kernels see it.
@@ -69,11 +70,17 @@ constexpr size_t kDescBlobSmall = 3840;
 constexpr size_t kDescBlobBytes = 16384;
 cudaError_t launch_store_blob(const void* host_bytes, size_t bytes, uint8_t* dst, int n_rope_chunks, const double* inv_freq,
                               int half_d, float2* cs_table, bool pdl, cudaStream_t st);
-// launch_assemble: acc != NULL fuses the deviation sums (which: bit 0 keys, bit 1 values) into the stitch.
+// launch_assemble: acc != NULL fuses the deviation sums (which: bit 0 keys, bit 1 values) into the stitch;
+// norm_sums != NULL ([n_chunks][L][assemble_parts_per_layer] doubles) also takes the key rows' norm sums,
+// which launch_importance_finalize turns into the chunks' importance scores (ChunkDesc::imp_out).
 cudaError_t launch_rope_table(const ChunkDesc* chunks, int n_chunks, const double* inv_freq, int half_d,
                               float2* cs_table, cudaStream_t st);
 cudaError_t launch_assemble(const ChunkDesc* chunks, int n_chunks, const float2* cs_table, const ModelDims& m,
-                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, bool pdl, cudaStream_t st);
+                            size_t smem_bytes, uint32_t* status, int which, unsigned long long* acc, double* norm_sums,
+                            bool pdl, cudaStream_t st);
+int assemble_parts_per_layer(int Hkv);
+cudaError_t launch_importance_finalize(const ChunkDesc* chunks, int n_chunks, const ModelDims& m, const double* norm_sums,
+                                       cudaStream_t st);
 size_t assemble_smem_bytes(const ModelDims& m, int mode);
 cudaError_t assemble_configure(size_t max_smem);
 

@@ -63,3 +63,66 @@ def test_chunk_importance_matches_oracle(kv_dtype, Hkv, Hq):
             assert np.abs(got - want).max() <= 1e-5 * np.abs(want).max()
     finally:
         B.kvb_destroy(ctx)
+
+
+@pytest.mark.parametrize("case", ["cfg0", "cfg1_L3", "mixed_bf16_H2", "mixed_fp16_H4", "mixed_bf16_H1"])
+def test_importance_as_a_by_product_of_the_stitch(case):
+    """kvb_request.importance: the stitching calls deliver Eq. 7 from the key rows they hold in
+    registers.  Against the oracle's fp64 value on the buffer the same call wrote (1e-6 relative),
+    identical from the one-pass call, the plain stitch and a repeated call (bit for bit: the norm sums
+    are added in a fixed order), and the stitched buffer and the selection are not disturbed."""
+    build_library()
+    from test_gpu_parity import _mixed_workload
+
+    if case == "cfg0":
+        wl = synth.workload(0)
+    elif case == "cfg1_L3":
+        w1 = synth.workload(1)
+        wl = synth.Workload(w1.name, w1.seed, synth.Shape(L=3), w1.requests, w1.select)
+    else:
+        kv_dtype, H = case.split("_")[1], int(case.split("_H")[1])
+        wl = _mixed_workload(H, 8, kv_dtype)
+    sh, sp = wl.shape, wl.select
+    reqs = prepare(wl)
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        Ts = [r.plan.T for r in reqs]
+        ks = [B.kvb_select_count(T, sp.ratio) for T in Ts]
+        # reference run without the importance output
+        tbl0 = B.RequestTable(reqs)
+        sel0 = B.SelectionTable(Ts, ks, [r.sel_capacity for r in reqs], DEV)
+        B.kvb_assemble_select(ctx, tbl0, sp.ratio, -1, sp.seam_before, sp.seam_after, sp.which, sel0)
+        B.kvb_last_status(ctx)
+        kv0 = [r.kv_buf.view(torch.int16).clone() for r in reqs]
+        got = {}
+        for call in ("one_pass", "one_pass_again", "stitch_only", "keys_not_compared"):
+            for r in reqs:
+                r.importance = torch.full((len(r.chunks),), -1.0, dtype=torch.float32, device=DEV)
+                r.kv_buf.zero_()
+            tbl = B.RequestTable(reqs)
+            sel = B.SelectionTable(Ts, ks, [r.sel_capacity for r in reqs], DEV)
+            if call == "stitch_only":
+                B.kvb_assemble(ctx, tbl)
+            else:  # which = 2: the deviation looks at values only, the key norms are still wanted
+                B.kvb_assemble_select(ctx, tbl, sp.ratio, -1, sp.seam_before, sp.seam_after, 2 if call == "keys_not_compared" else sp.which, sel)
+            B.kvb_last_status(ctx)
+            got[call] = [r.importance.clone() for r in reqs]
+            for r, k0 in zip(reqs, kv0):
+                assert torch.equal(r.kv_buf.view(torch.int16), k0)
+            if call == "one_pass":
+                for i in range(len(reqs)):
+                    assert torch.equal(sel.delta[i], sel0.delta[i]) and torch.equal(sel.sel[i], sel0.sel[i]) and torch.equal(sel.rank[i], sel0.rank[i])
+        for i, r in enumerate(reqs):
+            want = oracle.importance(helpers.bits_of(r.kv_buf), sh.C, helpers.dt_code(sh))
+            g = got["one_pass"][i].cpu().numpy().astype(np.float64)
+            assert np.abs(g - want).max() <= 1e-6 * np.abs(want).max(), np.abs(g / want - 1).max()
+            for other in ("one_pass_again", "stitch_only", "keys_not_compared"):
+                assert torch.equal(got["one_pass"][i], got[other][i]), other
+        # the stand-alone call on the stitched buffer agrees as well
+        outs = [torch.zeros(len(r.chunks), dtype=torch.float32, device=DEV) for r in reqs]
+        B.kvb_chunk_importance(ctx, B.RequestTable(reqs), outs)
+        B.kvb_last_status(ctx)
+        for i in range(len(reqs)):
+            assert float((outs[i] - got["one_pass"][i]).abs().max()) <= 2e-6 * float(outs[i].abs().max())
+    finally:
+        B.kvb_destroy(ctx)

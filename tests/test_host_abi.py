@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported():
 
 def test_struct_sizes_match_the_header_layout():
     assert C.sizeof(B.kvb_chunk) == 64 + 6 * 4 + 4 * 8
-    assert C.sizeof(B.kvb_request) == 8 + 3 * 8
+    assert C.sizeof(B.kvb_request) == 8 + 4 * 8
     assert C.sizeof(B.kvb_model_desc) == 8 * 4 + 8
     assert C.sizeof(B.kvb_selection) == 4 * 8 + 8
 
