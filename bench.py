@@ -126,8 +126,8 @@ class Replica:
 
     def __init__(self, B, ctx, wl, dev, seed_shift, meta_fp16=False):
         wl = synth.Workload(wl.name, wl.seed + 7919 * seed_shift, wl.shape, wl.requests, wl.select, wl.sigma_bulk, wl.sigma_seam, wl.seam_tokens)
-        qk, qv = B.quantize_fns(ctx, wl.shape, meta_fp16)
-        self.reqs = synth.materialize(wl, dev, qk, qv, B.assemble_fn(ctx))
+        bq = B.BatchedQuantizer(ctx, wl.shape, meta_fp16)  # the chunks of a request are quantised by one call
+        self.reqs = synth.materialize(wl, dev, bq.quantize_k, bq.quantize_v, bq.assemble)
         for r in self.reqs:
             for ck in r.chunks:
                 ck.meta_fp16 = int(ck.k_meta is not None and ck.k_meta.dtype == torch.float16)
@@ -576,6 +576,9 @@ class Runner:
         sh, sp = wl.shape, wl.select
         ctx, reps = self.build(key, wl)
         n_rep = len(reps)
+        B.kvb_destroy(ctx)  # a context sized for the stage's own calls (128 quantise jobs)
+        n_chunks = max(128, sum(len(r.chunks) for r in wl.requests))
+        ctx = B.create_for_shape(sh, self.local, max_requests=len(wl.requests), max_chunks_total=n_chunks, max_tokens_total=sum(r.T for r in wl.requests))
         for rep in reps:  # the selection and the stitched buffer the stage works on
             B.kvb_assemble_select(ctx, rep.tbl, sp.ratio, sp.k_override, sp.seam_before, sp.seam_after, sp.which, rep.sel)
         B.kvb_last_status(ctx)
@@ -591,6 +594,25 @@ class Runner:
             alg = sum(r.plan.T for r in reps[0].reqs) * sh.L * row_bytes  # every key row once
             call = lambda rep: B.kvb_chunk_importance(ctx, rep.tbl, rep.imp)
             passage = "Eq. 7 (kvb_chunk_importance)"
+        elif stage == "quantize":
+            # cache population of 128 chunks (a 16K-token prompt), keys and values, int8, one call
+            n_jobs = 128
+            g = torch.Generator(device=self.dev).manual_seed(5)
+            for rep in reps:
+                rep.qjobs = []
+                for _ in range(n_jobs):
+                    kx = torch.randn((sh.L, sh.C, sh.Hkv, sh.d), generator=g, device=self.dev).to(sh.torch_dtype)
+                    vx = torch.randn((sh.L, sh.C, sh.Hkv, sh.d), generator=g, device=self.dev).to(sh.torch_dtype)
+                    mk = lambda *shape: torch.empty(shape, dtype=torch.uint8, device=self.dev)
+                    rep.qjobs.append(dict(k=kx, v=vx, k_codes=mk(sh.L, sh.C, sh.Hkv, sh.d), v_codes=mk(sh.L, sh.C, sh.Hkv, sh.d),
+                                          k_meta=torch.empty((sh.L, 1, sh.Hkv, sh.d, 2), device=self.dev),
+                                          v_meta=torch.empty((sh.L, sh.C, sh.Hkv, 1, 2), device=self.dev), bits=8))
+            E = sh.Hkv * sh.d
+            alg = n_jobs * sh.L * (2 * sh.C * E * 2 + 2 * sh.C * E + E * 8 + sh.C * sh.Hkv * 8)  # 16-bit rows read, codes and metadata written
+            for rep in reps:
+                rep.qtable = B.QuantizeTable(rep.qjobs)  # marshalled once, like the request tables
+            call = lambda rep: B.kvb_quantize_chunks(ctx, rep.qtable)
+            passage = "Eq. 6 forward (kvb_quantize_chunks), %d chunks x (keys + values), int8" % n_jobs
         else:
             raise SystemExit("unknown stage %s" % stage)
         for i in range(max(args.warmup, 3)):
@@ -635,7 +657,7 @@ def main():
     ap.add_argument("--impl", default="kvb", choices=["kvb", "reference"])
     ap.add_argument("--workload", default="all", choices=["all"] + sorted(WORKLOADS),
                     help="all: the ragged batch (cfg4) as the headline plus cfg1, cfg2, cfg3 under per_config; or one workload alone")
-    ap.add_argument("--stage", default="path", choices=["path", "patch", "importance"], help="time one kernel next to the path instead of the path")
+    ap.add_argument("--stage", default="path", choices=["path", "patch", "importance", "quantize"], help="time one kernel next to the path instead of the path")
     ap.add_argument("--replicas", type=int, default=0, help="independent copies rotated through (0 = auto)")
     ap.add_argument("--batch", type=int, default=1, help="requests per step: the workload's request list repeated this many times")
     ap.add_argument("--requests", type=int, default=0, help="cfg4 only: the ragged batch's first N requests instead of all 32")

@@ -238,6 +238,29 @@ int kvb_quantize_keys_at(kvb_ctx* ctx, const void* x, int orig_pos, int bits, vo
 int kvb_quantize_chunk_ex(kvb_ctx* ctx, const void* x, int is_value, int bits, int unrotate_from, int meta_fp16,
                           void* codes, void* meta, void* cuda_stream);
 
+/* One chunk of a batched quantisation (host memory; all pointers device, 16-byte
+ * aligned).  k / v: the chunk's keys / values [L][C][H][d] in kv_dtype, NULL for
+ * a side that is not wanted; the outputs of a wanted side are required. */
+typedef struct {
+  const void* k;
+  const void* v;
+  void* k_codes;
+  void* v_codes;
+  void* k_meta;
+  void* v_meta;
+  int32_t bits;          /* 4 or 8 */
+  int32_t unrotate_from; /* < 0: keys as they are; >= 0: keys rotated back from that position first */
+  int32_t meta_fp16;     /* 1: compact (binary16) metadata */
+  int32_t reserved;
+} kvb_quantize_job;
+
+/* KV Quantization, Eq. 6, for a batch of chunks in one launch (cache population
+ * after a prefill: the Inference Engine's warm step stores every chunk of the
+ * prompt).  Each job is kvb_quantize_chunk_ex for the keys and / or the values of
+ * one chunk, with the same bit-exact code decision.  A context takes at least
+ * max_chunks_total jobs per call (KVB_ERR_WORKSPACE beyond its descriptor arena). */
+int kvb_quantize_chunks(kvb_ctx* ctx, const kvb_quantize_job* jobs, int n_jobs, void* cuda_stream);
+
 /* Cosine deviation of ONE request for callers that cannot allocate GPU memory:
  * a server that gave the whole GPU to its own block pool at start-up, or a
  * latency-critical thread that may not take the device-wide synchronisation an

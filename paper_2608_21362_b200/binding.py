@@ -77,6 +77,14 @@ class kvb_selection(C.Structure):
     ]
 
 
+class kvb_quantize_job(C.Structure):
+    _fields_ = [
+        ("k", C.c_void_p), ("v", C.c_void_p), ("k_codes", C.c_void_p), ("v_codes", C.c_void_p),
+        ("k_meta", C.c_void_p), ("v_meta", C.c_void_p),
+        ("bits", C.c_int32), ("unrotate_from", C.c_int32), ("meta_fp16", C.c_int32), ("reserved", C.c_int32),
+    ]
+
+
 class KvbError(RuntimeError):
     def __init__(self, status: int, message: str):
         super().__init__("kvb status %d (%s): %s" % (status, kvb_status_string(status), message))
@@ -286,6 +294,32 @@ def kvb_quantize_chunk_ex(ctx, x: torch.Tensor, is_value: bool, bits: int, unrot
     return _check(ctx, st) if check else st
 
 
+class QuantizeTable:
+    """Host-side kvb_quantize_job array built once from tensors and reusable across calls.
+    jobs: dicts with k / v (tensors or None), k_codes, v_codes, k_meta, v_meta (tensors), bits, and
+    optionally unrotate_from (default -1) and meta_fp16 (default False)."""
+
+    def __init__(self, jobs: Sequence[dict]):
+        self.n = len(jobs)
+        self._keep = list(jobs)
+        self.array = (kvb_quantize_job * max(self.n, 1))()
+        for a, j in zip(self.array, jobs):
+            for name in ("k", "v", "k_codes", "v_codes", "k_meta", "v_meta"):
+                t = j.get(name)
+                if t is not None:
+                    setattr(a, name, t.data_ptr())
+            a.bits, a.unrotate_from, a.meta_fp16 = int(j["bits"]), int(j.get("unrotate_from", -1)), int(j.get("meta_fp16", False))
+
+
+def kvb_quantize_chunks(ctx, jobs, stream=None, check: bool = True) -> int:
+    """jobs: a QuantizeTable, or a list of job dicts (marshalled on the spot)."""
+    L = lib()
+    L.kvb_quantize_chunks.argtypes = [C.c_void_p, C.POINTER(kvb_quantize_job), C.c_int, C.c_void_p]
+    tbl = jobs if isinstance(jobs, QuantizeTable) else QuantizeTable(jobs)
+    st = L.kvb_quantize_chunks(ctx, tbl.array, tbl.n, _stream(stream))
+    return _check(ctx, st) if check else st
+
+
 def kvb_deviation_static(device: int, model: kvb_model_desc, kv_buf: torch.Tensor, fresh: torch.Tensor, T: int,
                          which: int, delta: torch.Tensor, stream=None) -> int:
     """Deviation of one request without a context and without any allocation (static device scratch,
@@ -344,6 +378,51 @@ def quantize_fns(ctx, sh, meta_fp16: bool = False):
         return codes, meta
 
     return (lambda x, bits, group: _q(x, bits, False)), (lambda x, bits, group: _q(x, bits, True))
+
+
+class BatchedQuantizer:
+    """quantize_k / quantize_v / assemble callables in the form synth.materialize expects, with the
+    chunks of a request quantised by ONE kvb_quantize_chunks call: the quantise callables only allot
+    the outputs and note the job, the assemble callable (which materialize calls once per request,
+    after all its chunks) runs the batch before it stitches."""
+
+    def __init__(self, ctx, sh, meta_fp16: bool = False):
+        self.ctx, self.sh, self.meta_fp16, self.jobs = ctx, sh, meta_fp16, []
+        self._stitch = assemble_fn(ctx)
+
+    def _note(self, x: torch.Tensor, bits: int, is_value: bool):
+        sh = self.sh
+        mt = torch.float16 if self.meta_fp16 else torch.float32
+        L, Cn, H, d = x.shape
+        x = x.contiguous()
+        codes = torch.empty((L, Cn, H, d * bits // 8), dtype=torch.uint8, device=x.device)
+        if is_value:
+            meta = torch.empty((L, Cn, H, 1 if bits == 8 else d // sh.int4_group, 2), dtype=mt, device=x.device)
+            job = dict(v=x, v_codes=codes, v_meta=meta)
+            if self.jobs and "v" not in self.jobs[-1] and self.jobs[-1]["bits"] == bits:
+                self.jobs[-1].update(job)  # the values of the chunk whose keys were just noted: one job
+            else:
+                self.jobs.append(dict(job, bits=bits, meta_fp16=self.meta_fp16))
+        else:
+            meta = torch.empty((L, 1 if bits == 8 else Cn // sh.int4_group, H, d, 2), dtype=mt, device=x.device)
+            self.jobs.append(dict(k=x, k_codes=codes, k_meta=meta, bits=bits, meta_fp16=self.meta_fp16))
+        return codes, meta
+
+    def quantize_k(self, x, bits, group):
+        return self._note(x, bits, False)
+
+    def quantize_v(self, x, bits, group):
+        return self._note(x, bits, True)
+
+    def flush(self):
+        if self.jobs:
+            kvb_quantize_chunks(self.ctx, self.jobs)
+            kvb_last_status(self.ctx)
+            self.jobs = []
+
+    def assemble(self, sh, plan, chunks, fresh):
+        self.flush()
+        return self._stitch(sh, plan, chunks, fresh)
 
 
 def assemble_fn(ctx):

@@ -246,6 +246,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, assemble_configure(smem_max));
   KVB_CUDA(c, topk_configure());
   KVB_CUDA(c, attention_tc_configure());
+  KVB_CUDA(c, quantize_configure());
 
   const int half = m.d / 2;
   std::vector<double> inv(half);
@@ -257,6 +258,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   const size_t a1 = sizeof(ChunkDesc) * (size_t)limits->max_chunks_total;
   const size_t a2 = (sizeof(ReqDesc) + 256) * (size_t)limits->max_requests + 384 + sizeof(SeamWindow) * (size_t)limits->max_chunks_total;
   c->arena_bytes = ((a1 + 255) & ~(size_t)255) + ((a2 + 255) & ~(size_t)255);  // the fused call uploads both tables
+  static_assert(sizeof(QuantJob) <= sizeof(ChunkDesc), "a quantise job per chunk fits the chunk table's space");
   KVB_CUDA(c, cudaMalloc(&c->arena_dev, c->arena_bytes));
   KVB_CUDA(c, cudaMallocHost(&c->staging, c->arena_bytes * kSlots));
   for (int s = 0; s < kSlots; ++s) KVB_CUDA(c, cudaEventCreateWithFlags(&c->slot_done[s], cudaEventDisableTiming));
@@ -695,21 +697,55 @@ int kvb_chunk_importance(kvb_ctx* c, const kvb_request* reqs, int n_req, float* 
   return KVB_OK;
 }
 
+int kvb_quantize_chunks(kvb_ctx* c, const kvb_quantize_job* jobs, int n_jobs, void* cuda_stream) {
+  if (!c) return KVB_ERR_INVALID_ARG;
+  if (n_jobs < 0 || (n_jobs > 0 && !jobs)) return fail(c, KVB_ERR_INVALID_ARG, "bad job array");
+  if (n_jobs == 0) return KVB_OK;
+  if ((size_t)n_jobs * sizeof(QuantJob) > c->arena_bytes)
+    return fail(c, KVB_ERR_WORKSPACE, "%d jobs exceed the context's descriptor arena (%zu bytes)", n_jobs, c->arena_bytes);
+  for (int i = 0; i < n_jobs; ++i) {
+    const kvb_quantize_job& j = jobs[i];
+    if ((!j.k && !j.v) || (j.bits != 4 && j.bits != 8) || (j.meta_fp16 != 0 && j.meta_fp16 != 1))
+      return fail(c, KVB_ERR_INVALID_ARG, "job %d: bad quantize arguments", i);
+    if (j.unrotate_from >= (1 << 24)) return fail(c, KVB_ERR_INVALID_ARG, "job %d: position %d out of range [0, 2^24)", i, j.unrotate_from);
+    if ((j.k && (!j.k_codes || !j.k_meta)) || (j.v && (!j.v_codes || !j.v_meta)))
+      return fail(c, KVB_ERR_INVALID_ARG, "job %d: NULL output", i);
+    const void* ptrs[6] = {j.k, j.v, j.k_codes, j.v_codes, j.k_meta, j.v_meta};
+    for (const void* p : ptrs)
+      if (p && !aligned16(p)) return fail(c, KVB_ERR_BAD_TABLE, "job %d: quantize buffers must be 16-byte aligned", i);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  KVB_CUDA(c, cudaSetDevice(c->device));
+  uint8_t* host = nullptr;
+  const int slot_code = take_slot(c, &host);
+  if (slot_code >= 0) return slot_code;
+  const int slot = -slot_code - 1;
+  QuantJob* qj = reinterpret_cast<QuantJob*>(host);
+  for (int i = 0; i < n_jobs; ++i) {
+    const kvb_quantize_job& j = jobs[i];
+    qj[i] = QuantJob{j.k, j.v, j.k_codes, j.v_codes, j.k_meta, j.v_meta, j.bits, j.unrotate_from, j.meta_fp16, 0};
+  }
+  const int up = upload(c, slot, host, sizeof(QuantJob) * (size_t)n_jobs, st);
+  if (up != KVB_OK) return up;
+  c->last_stream = st;
+  KVB_CUDA(c, launch_quantize_batch(reinterpret_cast<const QuantJob*>(c->arena_dev), n_jobs, c->dims, c->inv_freq, c->status_dev, st));
+  c->launches += 1;
+  return KVB_OK;
+}
+
 int kvb_quantize_chunk_ex(kvb_ctx* c, const void* x, int is_value, int bits, int unrotate_from, int meta_fp16, void* codes,
                           void* meta, void* cuda_stream) {
   if (!c) return KVB_ERR_INVALID_ARG;
-  if (!x || !codes || !meta || (bits != 4 && bits != 8) || (meta_fp16 != 0 && meta_fp16 != 1))
-    return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");
+  if (!x || !codes || !meta) return fail(c, KVB_ERR_INVALID_ARG, "bad quantize arguments");
   if (unrotate_from >= 0 && is_value) return fail(c, KVB_ERR_INVALID_ARG, "values are never rotated");
-  if (unrotate_from >= (1 << 24)) return fail(c, KVB_ERR_INVALID_ARG, "position %d out of range [0, 2^24)", unrotate_from);
-  if (!aligned16(x) || !aligned16(codes) || !aligned16(meta)) return fail(c, KVB_ERR_BAD_TABLE, "quantize buffers must be 16-byte aligned");
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  KVB_CUDA(c, cudaSetDevice(c->device));
-  c->last_stream = st;
-  KVB_CUDA(c, launch_quantize(x, is_value ? 1 : 0, bits, codes, meta, c->dims, unrotate_from >= 0, unrotate_from >= 0 ? unrotate_from : 0,
-                              c->inv_freq, meta_fp16, st));
-  c->launches += 1;
-  return KVB_OK;
+  kvb_quantize_job j{};
+  (is_value ? j.v : j.k) = x;
+  (is_value ? j.v_codes : j.k_codes) = codes;
+  (is_value ? j.v_meta : j.k_meta) = meta;
+  j.bits = bits;
+  j.unrotate_from = unrotate_from;
+  j.meta_fp16 = meta_fp16;
+  return kvb_quantize_chunks(c, &j, 1, cuda_stream);
 }
 
 int kvb_quantize_chunk(kvb_ctx* c, const void* x, int is_value, int bits, void* codes, void* meta, void* cuda_stream) {

@@ -109,8 +109,22 @@ cudaError_t launch_patch(const ReqDesc* reqs, int n_req, int total_tiles, int ro
                          cudaStream_t st);
 cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, cudaStream_t st);
 
-// unrotate != 0 (keys only): rotate by R^(-orig_pos) before quantising (inv_freq: [d/2] doubles, device)
-cudaError_t launch_quantize(const void* x, int is_value, int bits, void* codes, void* meta, const ModelDims& m,
-                            int unrotate, int orig_pos, const double* inv_freq, int meta16, cudaStream_t st);
+// One chunk to quantise (device memory).  k / v NULL: that side is not wanted.
+struct QuantJob {
+  const void* k;
+  const void* v;
+  void* k_codes;
+  void* v_codes;
+  void* k_meta;
+  void* v_meta;
+  int32_t bits;
+  int32_t unrotate_from;  // >= 0 (keys only): rotate back by R^(-unrotate_from) before quantising
+  int32_t meta16;
+  int32_t reserved;
+};
+// inv_freq: [d/2] doubles, device
+cudaError_t launch_quantize_batch(const QuantJob* jobs, int n_jobs, const ModelDims& m, const double* inv_freq,
+                                  uint32_t* status, cudaStream_t st);
+cudaError_t quantize_configure();
 
 }  // namespace kvb

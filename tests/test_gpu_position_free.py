@@ -101,3 +101,66 @@ def test_reuse_at_another_position_is_one_rotation():
             assert np.all(np.abs(got[l] - want) <= bound)
     finally:
         B.kvb_destroy(ctx)
+
+
+@pytest.mark.parametrize("kv_dtype,Hkv", [("bf16", 2), ("fp16", 1), ("bf16", 4), ("fp16", 8)])
+def test_batched_quantiser_codes_bit_exact(kv_dtype, Hkv):
+    """kvb_quantize_chunks: one launch for a batch of chunks with mixed widths, keys only / values only
+    / both, keys rotated back or not, compact or float32 metadata.  Codes and metadata equal the
+    oracle's bit for bit (Eq. 6 forward: float32 subtract, divide, round-half-even on both sides),
+    including groups with tiny and with zero range, where the fast reciprocal must not decide."""
+    sh = synth.Shape(L=3, Hq=8, Hkv=Hkv, kv_dtype=kv_dtype)
+    dtc = helpers.dt_code(sh)
+    ctx = B.create_for_shape(sh, 0, max_chunks_total=16)
+    try:
+        specs = [  # (bits, keys?, values?, unrotate_from, meta_fp16)
+            (8, True, True, -1, False), (4, True, True, -1, False), (8, True, False, 4096 + 128, False), (4, True, True, 77, False),
+            (8, False, True, -1, False), (4, True, True, -1, True), (8, True, True, (1 << 24) - 128, True), (8, True, True, -1, False),
+        ]
+        jobs, xs = [], []
+        for i, (bits, has_k, has_v, pos, m16) in enumerate(specs):
+            k = _keys(sh, 100 + i)
+            v = _keys(sh, 200 + i)
+            if i == 7:  # degenerate groups: a constant channel, a constant row, a range of a few float32 ulps, a huge range
+                k[:, :, :, 3] = 1.25
+                v[:, 5] = -0.5
+                k[:, :, :, 9] = 1.0
+                k[:, 64:, :, 9] = 1.0 + 2.0 ** -7
+                v[:, 7, :, ::2] = 3.0e4 if kv_dtype == "fp16" else 1.0e30
+            mt = torch.float16 if m16 else torch.float32
+            j = dict(bits=bits, unrotate_from=pos, meta_fp16=m16)
+            if has_k:
+                j.update(k=k.to(DEV), k_codes=torch.zeros((sh.L, sh.C, Hkv, sh.d * bits // 8), dtype=torch.uint8, device=DEV),
+                         k_meta=torch.zeros((sh.L, 1 if bits == 8 else sh.C // sh.int4_group, Hkv, sh.d, 2), dtype=mt, device=DEV))
+            if has_v:
+                j.update(v=v.to(DEV), v_codes=torch.zeros((sh.L, sh.C, Hkv, sh.d * bits // 8), dtype=torch.uint8, device=DEV),
+                         v_meta=torch.zeros((sh.L, sh.C, Hkv, 1 if bits == 8 else sh.d // sh.int4_group, 2), dtype=mt, device=DEV))
+            jobs.append(j)
+            xs.append((k, v))
+        B.kvb_quantize_chunks(ctx, jobs)
+        B.kvb_last_status(ctx)
+        for (bits, has_k, has_v, pos, m16), j, (k, v) in zip(specs, jobs, xs):
+            gk, gv = (sh.C, sh.d) if bits == 8 else (sh.int4_group, sh.int4_group)
+            for l in range(sh.L):
+                if has_k:
+                    u = oracle.unrotate_keys(helpers.bits_of(k)[l], dtc, sh.theta, pos) if pos >= 0 else helpers.f64_of(k)[l]
+                    oc, om = oracle.quantize_k(u, bits, gk, meta16=m16)
+                    assert np.array_equal(j["k_codes"][l].cpu().numpy(), oc), ("key codes", bits, pos, m16)
+                    assert np.array_equal(j["k_meta"][l].float().cpu().numpy(), om.astype(np.float32)), ("key metadata", bits, pos, m16)
+                if has_v:
+                    oc, om = oracle.quantize_v(helpers.f64_of(v)[l], bits, gv, meta16=m16)
+                    assert np.array_equal(j["v_codes"][l].cpu().numpy(), oc), ("value codes", bits, m16)
+                    assert np.array_equal(j["v_meta"][l].float().cpu().numpy(), om.astype(np.float32)), ("value metadata", bits, m16)
+        # the one-chunk entry points are the same kernel with one job
+        c1 = torch.zeros_like(jobs[0]["k_codes"])
+        m1 = torch.zeros_like(jobs[0]["k_meta"])
+        B.kvb_quantize_chunk(ctx, jobs[0]["k"], False, 8, c1, m1)
+        B.kvb_last_status(ctx)
+        assert torch.equal(c1, jobs[0]["k_codes"]) and torch.equal(m1, jobs[0]["k_meta"])
+        # rejected: no side wanted, a missing output, too many jobs for the context
+        assert B.kvb_quantize_chunks(ctx, [dict(bits=8)], check=False) == B.KVB_ERR_INVALID_ARG
+        assert B.kvb_quantize_chunks(ctx, [dict(bits=8, k=jobs[0]["k"], k_codes=c1)], check=False) == B.KVB_ERR_INVALID_ARG
+        assert B.kvb_quantize_chunks(ctx, [jobs[0]] * 4096, check=False) == B.KVB_ERR_WORKSPACE
+        assert B.kvb_quantize_chunks(ctx, []) == B.KVB_OK
+    finally:
+        B.kvb_destroy(ctx)
