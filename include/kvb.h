@@ -317,7 +317,12 @@ int64_t kvb_launch_count(kvb_ctx* ctx);
  *                                 the pinned staging ring and cudaMemcpyAsync
  *   "attention_one_tile_per_cta"  default 0; 1 runs kvb_selective_attn with one tile
  *                                 per CTA instead of persistent CTAs
- * Every setting computes the same results; the tests compare them bit for bit.
+ *   "attention_cta_pairs"         default 0; 1 runs kvb_selective_attn on pairs of CTAs
+ *                                 (two neighbouring tiles on two SMs per MMA, keys by
+ *                                 sub-blocks of 128): measured slower than the default
+ *                                 form, kept as a cross-check; same result to the
+ *                                 attention tolerance, not bit for bit
+ * The first three settings compute the same bits; the tests compare them.
  * Unknown key or value: KVB_ERR_INVALID_ARG. */
 int kvb_set_debug_option(kvb_ctx* ctx, const char* key, int value);
 

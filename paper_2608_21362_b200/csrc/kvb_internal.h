@@ -105,6 +105,12 @@ cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req
                                 float scale, uint32_t* status, unsigned int* tile_counter, int n_sm, bool persistent,
                                 bool pdl, cudaStream_t st);
 
+// The paired form (csrc/attention_pair.cu): two tiles of one plane on two SMs per MMA.  total_pairs counts the
+// call's tile pairs over all requests and planes; ReqDesc::tile_offset counts a request's tile pairs per plane.
+cudaError_t attention_pair_configure();
+cudaError_t launch_attention_pair(const ReqDesc* reqs, const void* maps, int n_req, long long total_pairs, const ModelDims& m,
+                                  float scale, uint32_t* status, int n_sm, bool pdl, cudaStream_t st);
+
 cudaError_t launch_patch(const ReqDesc* reqs, int n_req, int total_tiles, int rows_per_cta, const ModelDims& m,
                          cudaStream_t st);
 cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, cudaStream_t st);

@@ -371,3 +371,38 @@ def test_selection_cluster_path_plateaus_windows_and_extremes():
                 assert n == len(want) and np.array_equal(sel.sel[i].cpu().numpy()[:n], want), (T, k)
     finally:
         B.kvb_destroy(ctx)
+
+
+def test_attention_cta_pair_form_matches_oracle():
+    """The paired form of the attention kernel (two neighbouring tiles on two SMs per MMA, the context's
+    "attention_cta_pairs" option; the single-CTA kernel is the default because it measures faster) computes
+    the same attention: against the oracle at 2e-2 on a batch whose tiles are short, ragged, odd in number
+    per plane and partly empty, with rows past n_sel left untouched.  Its bits may differ from the
+    single-CTA kernel's: keys go by sub-blocks of 128 instead of 64, so the lazy reference maximum moves at
+    other places and the float32 sums are taken in another order."""
+    sh = synth.Shape(L=3, Hq=16, Hkv=2)
+    plans = [synth._request(T, sh.C, [synth.MODE_INT8] * (T // sh.C), [((5 * i) % (T // sh.C)) * sh.C for i in range(T // sh.C)]) for T in (128, 640, 1152, 256, 2176)]
+    wl = synth.Workload("pairs", 37, sh, plans, synth.SelectPlan(ratio=0.2, seam_before=8, seam_after=8))
+    reqs = prepare(wl)
+    ctx = B.create_for_shape(sh, 0, max_requests=len(reqs))
+    try:
+        B.kvb_set_debug_option(ctx, "attention_cta_pairs", 1)
+        tbl = run_assemble(ctx, reqs)
+        Ts = [r.plan.T for r in reqs]
+        ks = [B.kvb_select_count(T, 0.2) for T in Ts]
+        sel = B.SelectionTable(Ts, ks, Ts, DEV)  # capacity T: many tiles past n_sel have no rows
+        for r in reqs:
+            r.sel_capacity = r.plan.T
+        B.kvb_deviation_topk(ctx, tbl, 0.2, -1, 8, 8, 3, sel)
+        qs = [torch.randn(sh.L, T, sh.Hq, sh.d, device=DEV, generator=torch.Generator(DEV).manual_seed(T)).to(r.fresh.dtype) for T, r in zip(Ts, reqs)]
+        out = [torch.zeros_like(q) for q in qs]
+        for _ in range(2):
+            B.kvb_selective_attn(ctx, tbl, sel, qs, out, 1.0 / math.sqrt(sh.d))
+        B.kvb_last_status(ctx)
+        for i, r in enumerate(reqs):
+            n = int(sel.n_sel[i])
+            r.q = qs[i]
+            check_attention(sh, r, sel.sel[i].cpu().numpy()[:n], out[i], None, None)
+            assert not out[i][:, n:].any()
+    finally:
+        B.kvb_destroy(ctx)
