@@ -396,7 +396,7 @@ class Runner:
             if dist:
                 ms = max_over_ranks([ms], dist, self.dev)[0]
             regions.append(ms)
-            if sum(regions) >= MIN_REGION_MS or len(regions) >= 400:
+            if sum(regions) >= args.min_region_ms or len(regions) >= 400:
                 break
         t_wall = time.perf_counter() - t_wall0
         clocks = self.sampler.end()
@@ -620,7 +620,7 @@ class Runner:
         self.sync_all()
         self.sampler.begin()
         regions, it = [], 0
-        while sum(regions) < MIN_REGION_MS and len(regions) < 400:
+        while (not regions or sum(regions) < args.min_region_ms) and len(regions) < 400:
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             for _ in range(args.steps):
@@ -663,6 +663,8 @@ def main():
     ap.add_argument("--requests", type=int, default=0, help="cfg4 only: the ragged batch's first N requests instead of all 32")
     ap.add_argument("--path", default="one-pass", choices=["one-pass", "two-call"], help="kvb_assemble_select, or kvb_assemble + kvb_deviation_topk")
     ap.add_argument("--meta-fp16", action="store_true", help="cached chunks carry compact (binary16) scale/min pairs")
+    ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,
+                    help="a K-step region shorter than this is repeated until this much device time has passed (0: one region, for profiler runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
