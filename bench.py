@@ -242,7 +242,7 @@ def oracle_sample_ids(wl):
     return order[:4] if sum(r.T for r in wl.requests) > 20000 else order
 
 
-def config_dict(wl, path, meta_fp16, world, n_replicas):
+def config_dict(wl, path, meta_fp16, world, n_replicas, attention_pairs=False):
     """The `config` object of the JSON line; both arms (kvb and reference) print the same one."""
     sh, sp = wl.shape, wl.select
     cfg = {
@@ -252,6 +252,8 @@ def config_dict(wl, path, meta_fp16, world, n_replicas):
         "kv_heads": sh.Hkv, "head_dim": sh.d, "chunk_tokens": sh.C, "select_ratio": sp.ratio, "seam_window": [sp.seam_before, sp.seam_after],
         "parallelism": "replicas only (one independent stream of requests per GPU)" if world > 1 else "single GPU",
     }
+    if attention_pairs:
+        cfg["attention"] = "paired-CTA form (debug option attention_cta_pairs)"
     cfg["l2"] = "inputs larger than L2, no flush: %s" % ("the batch itself exceeds it" if n_replicas == 1 else "%d independent replicas of the batch rotated" % n_replicas)
     return cfg
 
@@ -350,6 +352,8 @@ class Runner:
         n_chunks = sum(len(r.chunks) for r in wl.requests)
         n_tok = sum(r.T for r in wl.requests)
         ctx = B.create_for_shape(wl.shape, self.local, max_requests=len(wl.requests), max_chunks_total=n_chunks, max_tokens_total=n_tok)
+        if args.attention_pairs:
+            B.kvb_set_debug_option(ctx, "attention_cta_pairs", 1)
         n_rep = args.replicas or REPLICAS[key]
         reps = [Replica(B, ctx, wl, self.dev, 100 * self.rank + i, args.meta_fp16) for i in range(n_rep)]
         if key == "cfg3":  # the buffer and the selection the attention runs on, prepared outside the timed region
@@ -665,6 +669,8 @@ def main():
     ap.add_argument("--meta-fp16", action="store_true", help="cached chunks carry compact (binary16) scale/min pairs")
     ap.add_argument("--min-region-ms", type=float, default=MIN_REGION_MS,
                     help="a K-step region shorter than this is repeated until this much device time has passed (0: one region, for profiler runs)")
+    ap.add_argument("--attention-pairs", action="store_true",
+                    help="run kvb_selective_attn in its paired-CTA form (the context's attention_cta_pairs option; measured slower, not the default)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -725,7 +731,7 @@ def main():
         "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": head["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if sh.kv_dtype == "bf16" else "fp16", "data": "synthetic",
-        "config": config_dict(wl, PATH_NAMES[ONE_PASS] if head_key != "cfg3" else "kvb_selective_attn", args.meta_fp16, world, args.replicas or REPLICAS[head_key]),
+        "config": config_dict(wl, PATH_NAMES[ONE_PASS] if head_key != "cfg3" else "kvb_selective_attn", args.meta_fp16, world, args.replicas or REPLICAS[head_key], args.attention_pairs),
         "resident": head["l2"],
         "roofline": head["roofline"], "stages": head["stages"], "regions": head["regions"],
         "instrumented_ms_per_step": head["instrumented_ms_per_step"], "gpu_launches": head["gpu_launches"],
