@@ -6,9 +6,12 @@
 // One launch quantises a batch of chunks: a CTA per (chunk, layer, K|V, pair of KV heads).
 //   keys    the CTA's [128 tokens][<= 2 heads][128 channels] tile is fetched into shared memory by
 //           bulk copies (four large ones where the tile is contiguous, i.e. up to two KV heads;
-//           one per token row otherwise); a thread owns one channel, walks its token groups
-//           twice (extremes, then codes) and leaves the codes in a shared-memory tile that the
-//           CTA writes out in 16-byte pieces.  With `unrotate` every key is first rotated back
+//           one per token row otherwise); a thread owns a PAIR of neighbouring channels and a
+//           part of the tokens (one four-byte load per token brings both values, the arithmetic
+//           runs on packed float32 pairs), walks its token groups twice (extremes, then codes;
+//           with one group per chunk the parts exchange their extremes through shared memory)
+//           and leaves the codes in a shared-memory tile that the CTA writes out in 16-byte
+//           pieces.  With `unrotate` every key is first rotated back
 //           by R_theta^(-orig_pos) (Rotary Positional Embeddings, Eq. 3), so that the stored
 //           chunk is position-free and re-use at new_pos needs the single rotation by new_pos;
 //           cos / sin come from a double-precision angle, the rotation itself is float32 in a
@@ -16,9 +19,11 @@
 //   values  the same tile, staged the same way; a warp per (token, head) row, 4 channels per lane.
 // The division of the code decision is the hardware reciprocal where that provably gives the
 // same integer (the quotient lies away from every half-integer) and the IEEE division otherwise,
-// decided per warp so that the common case carries no division at all.
+// decided per warp and batch of eight tokens so that the common case carries no division at all.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
+
+#include <type_traits>
 
 #include "kvb_internal.h"
 
@@ -61,33 +66,55 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                : "memory");
 }
 
-template <int DT>
-__device__ __forceinline__ float from16(uint32_t bits16) {
-  if (DT == KVB_DT_BF16) return __uint_as_float(bits16 << 16);
-  const __half_raw r{(unsigned short)bits16};
-  return __half2float(__half(r));
+// The code of a value: rint((v - mn) / s) clamped to [0, levels], the division being IEEE float32.
+// Fast form, on packed pairs of values: q = (v - mn) * (1/s) with the hardware reciprocal (at most
+// one unit in the last place off) differs from the real quotient by at most 1.5 * 2^-23 * q and the
+// IEEE quotient by at most 2^-24 * q: together 2.5 * 2^-23 * levels < 3e-7 * levels.  When q lies
+// further than 4e-7 * levels from every half-integer both therefore round to the same integer.
+// q + 2^23 rounds q to that integer (round-half-even, as rint does) and leaves it in the low mantissa
+// bits; no clamp is needed, the quotient cannot exceed levels by more than a rounding error.  The
+// distance of q from its integer, |q - rint(q)|, is exact in float32; the caller keeps its maximum
+// over a few values and lets the IEEE division decide for exactly those whose distance comes within
+// the bound of one half (about one value in five thousand for 8-bit codes).
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
 }
-
-// The code of one value: rint((v - mn) / s) clamped to [0, levels], the division being IEEE float32.
-// Fast form: q = (v - mn) * (1/s) with the hardware reciprocal is within 2e-7 * q <= 5e-5 of the exact
-// quotient, and so is the IEEE quotient (1.5e-5): when q lies further than 2.5e-4 from every
-// half-integer both round to the same integer.  q + 2^23 rounds q to that integer (round-half-even,
-// as rint does) and leaves it in the low mantissa bits; no clamp is needed, the quotient cannot
-// exceed levels by more than a rounding error.  `unsafe` tells the caller that the IEEE division must
-// decide instead (about one value in a thousand; NaN or infinite q as well).
-struct FastCode {
-  uint32_t code;
-  bool unsafe;
-};
-__device__ __forceinline__ FastCode code_fast(float v, float mn, float inv_s) {
-  const float t = __fsub_rn(v, mn);
-  const float q = t * inv_s;
-  const float m = __fadd_rn(q, 8388608.0f);
-  const float d = q - __fsub_rn(m, 8388608.0f);
-  FastCode r;
-  r.code = __float_as_uint(m) & 0x1FFu;
-  r.unsafe = !(fabsf(fabsf(d) - 0.5f) >= 2.5e-4f) || !(q <= 300.f);
-  return r;
+__device__ __forceinline__ void f2_unpack(uint64_t d, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(d)); }
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+constexpr float kMagic = 8388608.0f;  // 2^23
+// The value pair v2 against (mn2, inv2): m0 / m1 = rint(q) + 2^23 as floats (the code in the low
+// mantissa bits), r0 / r1 = rint(q); returns the larger |q - rint(q)| of the two.
+__device__ __forceinline__ float code_fast2(uint64_t v2, uint64_t mn2, uint64_t inv2, float& m0, float& m1, float& r0, float& r1) {
+  const uint64_t magic2 = f2_pack(kMagic, kMagic);
+  const uint64_t q2 = f2_mul(f2_sub(v2, mn2), inv2);
+  const uint64_t m2 = f2_add(q2, magic2);
+  const uint64_t r2 = f2_sub(m2, magic2);
+  float d0, d1;
+  f2_unpack(f2_sub(q2, r2), d0, d1);
+  f2_unpack(m2, m0, m1);
+  f2_unpack(r2, r0, r1);
+  return fmaxf(fabsf(d0), fabsf(d1));
 }
 // not inlined: the compiler must not evaluate the division speculatively on the common path
 __device__ __noinline__ uint32_t code_exact(float v, float mn, float s, float levels) {
@@ -95,12 +122,58 @@ __device__ __noinline__ uint32_t code_exact(float v, float mn, float s, float le
   c = fminf(fmaxf(c, 0.f), levels);
   return (uint32_t)c;
 }
-// 1/s for code_fast; a scale too small for an accurate reciprocal gives NaN, which sends every value
-// of the group through the IEEE division
+// 1/s for code_fast2; usable: the scale is in the range where the reciprocal is accurate (otherwise
+// the IEEE division decides for the whole group)
 __device__ __forceinline__ float rcp_approx(float x) {
   float y;
   asm("rcp.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return x >= 1e-30f ? y : __int_as_float(0x7FC00000);
+  return y;
+}
+__device__ __forceinline__ bool scale_usable(float s) { return s >= 1e-30f && s <= 1e30f; }
+// largest |q - rint(q)| for which the fast code is trusted; below zero when the scale is not usable
+__device__ __forceinline__ float trust_limit(float s, float levels) { return scale_usable(s) ? 0.5f - 4e-7f * levels : -1.f; }
+
+// four codes, each in the low byte of m_i's bit pattern, as one word (code 0 in the lowest byte)
+__device__ __forceinline__ uint32_t pack4_u8(float m0, float m1, float m2, float m3) {
+  const uint32_t a = __byte_perm(__float_as_uint(m0), __float_as_uint(m1), 0x0040);
+  const uint32_t b = __byte_perm(__float_as_uint(m2), __float_as_uint(m3), 0x0040);
+  return __byte_perm(a, b, 0x5410);
+}
+// two 4-bit codes as one byte (code 0 in the low nibble), in the low mantissa bits of the result:
+// r1 * 16 + (r0 + 2^23), exact
+__device__ __forceinline__ float pack2_u4(float m0, float r1) { return fmaf(r1, 16.f, m0); }
+
+// two 16-bit values of one 32-bit word as a packed float32 pair
+template <int DT>
+__device__ __forceinline__ uint64_t unpack2(uint32_t w) {
+  if (DT == KVB_DT_BF16) return f2_pack(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+  const float2 t = __half22float2(*reinterpret_cast<const __half2*>(&w));
+  return f2_pack(t.x, t.y);
+}
+// element-wise minimum / maximum of two words of two 16-bit values each (exact: no rounding is involved)
+template <int DT>
+__device__ __forceinline__ uint32_t min2_16(uint32_t a, uint32_t b) {
+  uint32_t r;
+  if (DT == KVB_DT_BF16) {
+    const __nv_bfloat162 t = __hmin2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+    r = *reinterpret_cast<const uint32_t*>(&t);
+  } else {
+    const __half2 t = __hmin2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
+    r = *reinterpret_cast<const uint32_t*>(&t);
+  }
+  return r;
+}
+template <int DT>
+__device__ __forceinline__ uint32_t max2_16(uint32_t a, uint32_t b) {
+  uint32_t r;
+  if (DT == KVB_DT_BF16) {
+    const __nv_bfloat162 t = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&a), *reinterpret_cast<const __nv_bfloat162*>(&b));
+    r = *reinterpret_cast<const uint32_t*>(&t);
+  } else {
+    const __half2 t = __hmax2(*reinterpret_cast<const __half2*>(&a), *reinterpret_cast<const __half2*>(&b));
+    r = *reinterpret_cast<const uint32_t*>(&t);
+  }
+  return r;
 }
 
 // (scale, min) of a group from its extremes.  Compact metadata: min is rounded down to binary16
@@ -118,18 +191,22 @@ __device__ __forceinline__ void store_meta(float* meta, size_t pair, float s, fl
   }
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kThreads)
+template <int DT, int HP>  // HP: KV heads of a CTA's tile (1 or 2)
+__global__ void __launch_bounds__(kThreads, 3)
     quantize_batch_kernel(const QuantJob* __restrict__ jobs, ModelDims m, const double* __restrict__ inv_freq,
                           uint32_t* __restrict__ status) {
+  constexpr int W = HP * kD;            // channels of the tile
+  constexpr int NQ = W / 4;             // channel quads of the tile (keys: one thread each)
+  constexpr int kParts = kThreads / NQ; // keys: parts of the tokens (4 or 8)
+  constexpr int kTokPer = kTokens / kParts;  // keys: tokens of a part (32 or 16)
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ __align__(8) uint64_t bar;
+  __shared__ float4 s_mn[kThreads], s_mx[kThreads];  // keys: extremes of every (part, quad)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = m.Hkv;
-  const int hp = H < 2 ? 1 : 2;           // heads of this CTA's tile
-  const int n_hp = H / hp;
+  const int n_hp = H / HP;
   int item = blockIdx.x;
-  const int hb = (item % n_hp) * hp;      // first head
+  const int hb = (item % n_hp) * HP;      // first head
   item /= n_hp;
   const int kv = item & 1;
   const int l = (item >> 1) % m.L;
@@ -143,12 +220,10 @@ __global__ void __launch_bounds__(kThreads)
   const int E = H * kD;                   // elements of a token row
   const size_t layer_elems = (size_t)kTokens * E;
 
-  // ------------------------------ the tile [128 tokens][hp heads][128 channels] through shared memory,
+  // ------------------------------ the tile [128 tokens][HP heads][128 channels] into shared memory,
   //                                all of it in flight at once
-  const int W = hp * kD;                       // channels of the tile
-  const uint32_t row_bytes = (uint32_t)W * 2;  // one token row of the tile
-  uint16_t* s_x = reinterpret_cast<uint16_t*>(smem);                    // [128][W]
-  uint8_t* s_codes = smem + (size_t)kTokens * row_bytes;                // keys: [128][W * bits / 8]
+  constexpr uint32_t row_bytes = (uint32_t)W * 2;  // one token row of the tile
+  uint16_t* s_x = reinterpret_cast<uint16_t*>(smem);  // [128][W]
   const uint16_t* tile = x + (size_t)l * layer_elems + (size_t)hb * kD;
   if (tid == 0) {
     mbar_init(&bar, 1);
@@ -158,139 +233,285 @@ __global__ void __launch_bounds__(kThreads)
   if (warp == 0) {
     if (lane == 0) mbar_expect_tx(&bar, (uint32_t)kTokens * row_bytes);
     __syncwarp();
-    if (W == E) {  // up to two KV heads: the tile is one contiguous block -- four large copies
+    if (W == E) {  // the tile is one contiguous block -- four large copies
       if (lane < 4) bulk_g2s(s_x + (size_t)lane * (kTokens / 4) * W, tile + (size_t)lane * (kTokens / 4) * W, (uint32_t)(kTokens / 4) * row_bytes, &bar);
     } else {       // more heads: one copy per token row (the copy engine's request rate, not its bandwidth, sets the pace)
       for (int t = lane; t < kTokens; t += 32) bulk_g2s(s_x + (size_t)t * W, tile + (size_t)t * E, row_bytes, &bar);
     }
   }
-
-  if (kv) {
-    // ------------------------------ values: a warp per (token, head) row, 4 channels per lane
-    const int group_ch = bits == 8 ? kD : m.int4_group;
-    const int G = kD / group_ch;
-    const int lanes_per_group = group_ch / 4;  // 32 (int8, whole row) or 8 (groups of 32 channels)
-    const bool ok = mbar_wait(&bar, 0);
-    if (!ok) {
-      if (tid == 0) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
-      return;
-    }
-    for (int r = warp; r < kTokens * hp; r += kThreads / 32) {
-      const int t = r / hp, hh = r % hp;
-      const size_t u = (size_t)l * kTokens * H + (size_t)t * H + hb + hh;  // (layer, token, head) row
-      const uint2 w = *reinterpret_cast<const uint2*>(s_x + (size_t)t * W + hh * kD + 4 * lane);
-      float v[4] = {from16<DT>(w.x & 0xFFFFu), from16<DT>(w.x >> 16), from16<DT>(w.y & 0xFFFFu), from16<DT>(w.y >> 16)};
-      float mn = fminf(fminf(v[0], v[1]), fminf(v[2], v[3])), mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
-      for (int o = 1; o < lanes_per_group; o <<= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-      }
-      float s;
-      group_params(mn, mx, levels, jb.meta16, s);
-      const float inv_s = rcp_approx(s);
-      if ((lane % lanes_per_group) == 0) store_meta(meta, u * G + (4 * lane) / group_ch, s, mn, jb.meta16);
-      uint32_t q[4];
-      bool unsafe = false;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const FastCode f = code_fast(v[i], mn, inv_s);
-        q[i] = f.code;
-        unsafe |= f.unsafe;
-      }
-      if (__any_sync(0xffffffffu, unsafe)) {  // rare: the whole warp takes the IEEE division
-#pragma unroll
-        for (int i = 0; i < 4; ++i) q[i] = code_exact(v[i], mn, s, levels);
-      }
-      if (bits == 8) {
-        *reinterpret_cast<uint32_t*>(codes + u * kD + 4 * lane) = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
-      } else {
-        *reinterpret_cast<uint16_t*>(codes + ((u * kD) >> 1) + 2 * lane) = (uint16_t)(q[0] | (q[1] << 4) | (q[2] << 8) | (q[3] << 12));
-      }
-    }
+  const bool ok = __syncthreads_and(mbar_wait(&bar, 0));  // one answer for the whole CTA
+  if (!ok) {
+    if (tid == 0) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
     return;
   }
 
-  // ------------------------------ keys: a thread per channel of the tile
-  const int group_tokens = bits == 8 ? kTokens : m.int4_group;
-  const int G = kTokens / group_tokens;
-  const bool rot = jb.unrotate_from >= 0;
-  const int c = tid;  // channel of the tile (W <= kThreads)
-  float cs = 1.f, sn = 0.f;
-  int partner = c;
-  if (rot && c < W) {
-    const int j = c & 127;  // channel within the head; planes pair j with j + 64
-    double s_d, c_d;
-    sincos((double)jb.unrotate_from * inv_freq[j & 63], &s_d, &c_d);
-    cs = (float)c_d;
-    sn = j < 64 ? (float)s_d : -(float)s_d;  // low half: + x_hi * s; high half: - x_lo * s
-    partner = c ^ 64;
-  }
-  const bool ok = mbar_wait(&bar, 0);
-  if (!ok && tid == 0) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
-  if (ok && c < W) {
-    auto value = [&](int t) {
-      const float v = from16<DT>(s_x[(size_t)t * W + c]);
-      if (!rot) return v;
-      return fmaf(v, cs, __fmul_rn(from16<DT>(s_x[(size_t)t * W + partner]), sn));
-    };
-    const int h = hb + c / kD, j = c % kD;
-    for (int g = 0; g < G; ++g) {
-      float mn = INFINITY, mx = -INFINITY;
-#pragma unroll 8
-      for (int t = g * group_tokens; t < (g + 1) * group_tokens; ++t) {
-        const float v = value(t);
-        mn = fminf(mn, v);
-        mx = fmaxf(mx, v);
-      }
-      float s;
-      group_params(mn, mx, levels, jb.meta16, s);
-      const float inv_s = rcp_approx(s);
-      store_meta(meta, (((size_t)l * G + g) * H + h) * kD + j, s, mn, jb.meta16);
-#pragma unroll 8
-      for (int t = g * group_tokens; t < (g + 1) * group_tokens; ++t) {
-        const float v = value(t);
-        const FastCode f = code_fast(v, mn, inv_s);
-        uint32_t q = f.code;
-        if (__any_sync(0xffffffffu, f.unsafe)) q = code_exact(v, mn, s, levels);  // rare; whole warps are here
-        if (bits == 8) {
-          s_codes[(size_t)t * W + c] = (uint8_t)q;
-        } else {
-          const uint32_t other = __shfl_xor_sync(0xffffffffu, q, 1);  // W is a multiple of 32: whole warps are here
-          if ((c & 1) == 0) s_codes[((size_t)t * W + c) >> 1] = (uint8_t)(q | (other << 4));
+  if (kv) {
+    // ------------------------------ values: eight lanes per (token, head) row, a warp takes four rows at
+    // a time.  A lane holds two pieces of eight channels, 8 j .. 8 j + 7 and 64 + 8 j .. 64 + 8 j + 7
+    // (two conflict-free 16-byte loads); the extremes are taken on the 16-bit values, two per
+    // instruction, and reduced over the lanes of a group by shuffles of those words.
+    auto values = [&](auto bits_tag) {
+      constexpr int BITS = decltype(bits_tag)::value;
+      constexpr int G = BITS == 8 ? 1 : kD / 32;  // groups of a row: the whole row, or 32 channels each
+      const int sub = lane >> 3, lj = lane & 7;
+      for (int r = warp * 4 + sub; r < kTokens * HP; r += (kThreads / 32) * 4) {
+        const int t = r / HP, hh = r % HP;
+        const size_t u = ((size_t)l * kTokens + t) * H + hb + hh;  // (layer, token, head) row
+        const uint4 wa = *reinterpret_cast<const uint4*>(s_x + (size_t)r * kD + 8 * lj);
+        const uint4 wb = *reinterpret_cast<const uint4*>(s_x + (size_t)r * kD + 64 + 8 * lj);
+        const uint32_t w[2][4] = {{wa.x, wa.y, wa.z, wa.w}, {wb.x, wb.y, wb.z, wb.w}};
+        uint32_t lo[2], hi[2];  // per piece: element-wise extremes of its four words
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          lo[p] = min2_16<DT>(min2_16<DT>(w[p][0], w[p][1]), min2_16<DT>(w[p][2], w[p][3]));
+          hi[p] = max2_16<DT>(max2_16<DT>(w[p][0], w[p][1]), max2_16<DT>(w[p][2], w[p][3]));
+        }
+        if (G == 1) {  // one group: both pieces, all eight lanes
+          lo[0] = min2_16<DT>(lo[0], lo[1]);
+          hi[0] = max2_16<DT>(hi[0], hi[1]);
+        }
+        constexpr int kPieces = G == 1 ? 1 : 2;     // groups this lane takes part in
+        constexpr int kLanes = G == 1 ? 8 : 4;      // lanes of a group
+        float mn[2], s[2], limit[2];
+        uint64_t mn2[2], inv2[2];
+#pragma unroll
+        for (int p = 0; p < kPieces; ++p) {
+#pragma unroll
+          for (int o = 1; o < kLanes; o <<= 1) {
+            lo[p] = min2_16<DT>(lo[p], __shfl_xor_sync(0xffffffffu, lo[p], o));
+            hi[p] = max2_16<DT>(hi[p], __shfl_xor_sync(0xffffffffu, hi[p], o));
+          }
+          float a, b, c, d;
+          f2_unpack(unpack2<DT>(lo[p]), a, b);
+          f2_unpack(unpack2<DT>(hi[p]), c, d);
+          mn[p] = fminf(a, b);
+          group_params(mn[p], fmaxf(c, d), levels, jb.meta16, s[p]);
+          const int g = G == 1 ? 0 : 2 * p + (lj >> 2);  // channels 8 lj (+ 64) lie in group lj / 4 (+ 2)
+          if ((lj & (kLanes - 1)) == 0) store_meta(meta, u * G + g, s[p], mn[p], jb.meta16);
+          const float inv = rcp_approx(s[p]);
+          mn2[p] = f2_pack(mn[p], mn[p]);
+          inv2[p] = f2_pack(inv, inv);
+          limit[p] = trust_limit(s[p], levels);
+        }
+#pragma unroll
+        for (int p = 0; p < 2; ++p) {
+          const int pp = G == 1 ? 0 : p;
+          float mq[4][2], rq[4][2], dev[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dev[i] = code_fast2(unpack2<DT>(w[p][i]), mn2[pp], inv2[pp], mq[i][0], mq[i][1], rq[i][0], rq[i][1]);
+          uint32_t out[2];
+          if (BITS == 8) {
+            out[0] = pack4_u8(mq[0][0], mq[0][1], mq[1][0], mq[1][1]);
+            out[1] = pack4_u8(mq[2][0], mq[2][1], mq[3][0], mq[3][1]);
+          } else {
+            out[0] = pack4_u8(pack2_u4(mq[0][0], rq[0][1]), pack2_u4(mq[1][0], rq[1][1]), pack2_u4(mq[2][0], rq[2][1]),
+                              pack2_u4(mq[3][0], rq[3][1]));
+          }
+          const float worst = fmaxf(fmaxf(dev[0], dev[1]), fmaxf(dev[2], dev[3]));
+          if (__any_sync(0xffffffffu, worst > limit[pp])) {  // rare: the IEEE division decides for the words near a tie
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              if (dev[i] > limit[pp]) {
+                float a, b;
+                f2_unpack(unpack2<DT>(w[p][i]), a, b);
+                const uint32_t c0 = code_exact(a, mn[pp], s[pp], levels), c1 = code_exact(b, mn[pp], s[pp], levels);
+                if (BITS == 8) {
+                  const int sh = (i & 1) * 16;
+                  out[i >> 1] = (out[i >> 1] & ~(0xFFFFu << sh)) | ((c0 | (c1 << 8)) << sh);
+                } else {
+                  out[0] = (out[0] & ~(0xFFu << (8 * i))) | ((c0 | (c1 << 4)) << (8 * i));
+                }
+              }
+            }
+          }
+          if (BITS == 8)
+            *reinterpret_cast<uint2*>(codes + u * kD + 64 * p + 8 * lj) = make_uint2(out[0], out[1]);
+          else
+            *reinterpret_cast<uint32_t*>(codes + u * (kD / 2) + 32 * p + 4 * lj) = out[0];
         }
       }
-    }
+    };
+    if (bits == 8) values(std::integral_constant<int, 8>{});
+    else values(std::integral_constant<int, 4>{});
+    return;
   }
-  __syncthreads();
-  if (ok) {  // the code tile leaves in 16-byte pieces: a token row of the tile is contiguous in the layer's codes
-    const int row_code_bytes = W * bits / 8, pieces = row_code_bytes / 16;
-    uint8_t* out = codes + (((size_t)l * layer_elems + (size_t)hb * kD) * bits) / 8;
-    for (int i = tid; i < kTokens * pieces; i += kThreads) {
-      const int t = i / pieces, p = i % pieces;
-      *reinterpret_cast<uint4*>(out + (size_t)t * (E * bits / 8) + p * 16) =
-          *reinterpret_cast<const uint4*>(s_codes + (size_t)t * row_code_bytes + p * 16);
+
+  // ------------------------------ keys: a thread per QUAD of neighbouring channels and part of the tokens.
+  // One eight-byte load brings a token's four values; the extremes are taken on the 16-bit values
+  // (two per instruction; on the rotated float32 values with `unrotate`), subtract, scale and round
+  // run as packed float32 pairs, and a token's four codes leave with one store.
+  const int quad = tid % NQ;                 // tile channels 4 quad .. 4 quad + 3
+  const int part = tid / NQ;                 // tokens part * kTokPer .. + kTokPer - 1
+  const int c = 4 * quad;
+  const int h = hb + c / kD, j = c % kD;
+  const uint2* s_q = reinterpret_cast<const uint2*>(s_x);  // [128][NQ] words pairs of four channels
+
+  auto keys = [&](auto bits_tag, auto rot_tag) {
+    constexpr int BITS = decltype(bits_tag)::value;
+    constexpr bool ROT = decltype(rot_tag)::value;
+    constexpr int kGroupTokens = BITS == 8 ? kTokens : 32;  // one group per chunk, or groups of 32 tokens
+    constexpr int G = kTokens / kGroupTokens;
+    constexpr int kPartsPerGroup = kGroupTokens / kTokPer;
+    uint64_t cs2[2] = {0, 0}, sn2[2] = {0, 0};
+    if (ROT) {  // channel j pairs with j + 64: low half + x_hi * s, high half - x_lo * s
+      float cs[4], sn[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        double s_d, c_d;
+        sincos((double)jb.unrotate_from * inv_freq[(j + i) & 63], &s_d, &c_d);
+        cs[i] = (float)c_d;
+        sn[i] = j < 64 ? (float)s_d : -(float)s_d;
+      }
+      cs2[0] = f2_pack(cs[0], cs[1]), cs2[1] = f2_pack(cs[2], cs[3]);
+      sn2[0] = f2_pack(sn[0], sn[1]), sn2[1] = f2_pack(sn[2], sn[3]);
     }
+    // the four values of token t as two packed pairs
+    auto value4 = [&](int t, uint64_t& v01, uint64_t& v23) {
+      const uint2 w = s_q[t * NQ + quad];
+      v01 = unpack2<DT>(w.x), v23 = unpack2<DT>(w.y);
+      if (ROT) {  // per value: fma(x, c, x_partner * s), as the one-chunk form
+        const uint2 wp = s_q[t * NQ + (quad ^ 16)];
+        v01 = f2_fma(v01, cs2[0], f2_mul(unpack2<DT>(wp.x), sn2[0]));
+        v23 = f2_fma(v23, cs2[1], f2_mul(unpack2<DT>(wp.y), sn2[1]));
+      }
+    };
+    // ---- extremes of this part's tokens
+    const int t0 = part * kTokPer;
+    float mn[4], mx[4];
+    if (!ROT) {
+      uint2 lo = s_q[t0 * NQ + quad], hi = lo;
+#pragma unroll 8
+      for (int t = t0 + 1; t < t0 + kTokPer; ++t) {
+        const uint2 w = s_q[t * NQ + quad];
+        lo.x = min2_16<DT>(lo.x, w.x), lo.y = min2_16<DT>(lo.y, w.y);
+        hi.x = max2_16<DT>(hi.x, w.x), hi.y = max2_16<DT>(hi.y, w.y);
+      }
+      f2_unpack(unpack2<DT>(lo.x), mn[0], mn[1]);
+      f2_unpack(unpack2<DT>(lo.y), mn[2], mn[3]);
+      f2_unpack(unpack2<DT>(hi.x), mx[0], mx[1]);
+      f2_unpack(unpack2<DT>(hi.y), mx[2], mx[3]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) mn[i] = INFINITY, mx[i] = -INFINITY;
+#pragma unroll 4
+      for (int t = t0; t < t0 + kTokPer; ++t) {
+        uint64_t v01, v23;
+        value4(t, v01, v23);
+        float v[4];
+        f2_unpack(v01, v[0], v[1]);
+        f2_unpack(v23, v[2], v[3]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) mn[i] = fminf(mn[i], v[i]), mx[i] = fmaxf(mx[i], v[i]);
+      }
+    }
+    // ---- the parts of a group exchange their extremes
+    s_mn[part * NQ + quad] = make_float4(mn[0], mn[1], mn[2], mn[3]);
+    s_mx[part * NQ + quad] = make_float4(mx[0], mx[1], mx[2], mx[3]);
+    __syncthreads();
+    const int g = part / kPartsPerGroup;
+#pragma unroll
+    for (int q = 0; q < kPartsPerGroup; ++q) {
+      const float4 a = s_mn[(g * kPartsPerGroup + q) * NQ + quad], b = s_mx[(g * kPartsPerGroup + q) * NQ + quad];
+      mn[0] = fminf(mn[0], a.x), mn[1] = fminf(mn[1], a.y), mn[2] = fminf(mn[2], a.z), mn[3] = fminf(mn[3], a.w);
+      mx[0] = fmaxf(mx[0], b.x), mx[1] = fmaxf(mx[1], b.y), mx[2] = fmaxf(mx[2], b.z), mx[3] = fmaxf(mx[3], b.w);
+    }
+    float s[4], limit = 1.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      group_params(mn[i], mx[i], levels, jb.meta16, s[i]);
+      limit = fminf(limit, trust_limit(s[i], levels));
+    }
+    if (part % kPartsPerGroup == 0) {
+      const size_t pair = (((size_t)l * G + g) * H + h) * kD + j;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) store_meta(meta, pair + i, s[i], mn[i], jb.meta16);
+    }
+    // ---- codes, kBatch tokens at a time
+    constexpr int kBatch = 4;
+    const uint64_t mn01 = f2_pack(mn[0], mn[1]), mn23 = f2_pack(mn[2], mn[3]);
+    const uint64_t inv01 = f2_pack(rcp_approx(s[0]), rcp_approx(s[1])), inv23 = f2_pack(rcp_approx(s[2]), rcp_approx(s[3]));
+    const size_t row_stride = (size_t)E * BITS / 8;  // bytes of a token row of the layer's codes
+    uint8_t* out = codes + (((size_t)l * layer_elems + (size_t)hb * kD + c) * BITS) / 8 + (size_t)t0 * row_stride;
+    for (int t8 = t0; t8 < t0 + kTokPer; t8 += kBatch, out += kBatch * row_stride) {
+      uint32_t cw[kBatch];
+      float dev[kBatch], worst = 0.f;
+#pragma unroll
+      for (int i = 0; i < kBatch; ++i) {
+        uint64_t v01, v23;
+        value4(t8 + i, v01, v23);
+        float ma[2], mb[2], ra[2], rb[2];
+        dev[i] = fmaxf(code_fast2(v01, mn01, inv01, ma[0], ma[1], ra[0], ra[1]), code_fast2(v23, mn23, inv23, mb[0], mb[1], rb[0], rb[1]));
+        worst = fmaxf(worst, dev[i]);
+        if (BITS == 8)
+          cw[i] = pack4_u8(ma[0], ma[1], mb[0], mb[1]);
+        else
+          cw[i] = __float_as_uint(fmaf(pack2_u4(rb[0], rb[1]), 256.f, pack2_u4(ma[0], ra[1])));  // low 16 bits
+      }
+      if (__any_sync(0xffffffffu, worst > limit)) {  // rare: the IEEE division decides for the tokens near a tie
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+          if (dev[i] > limit) {
+            uint64_t v01, v23;
+            value4(t8 + i, v01, v23);
+            float v[4];
+            f2_unpack(v01, v[0], v[1]);
+            f2_unpack(v23, v[2], v[3]);
+            uint32_t w = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) w |= code_exact(v[e], mn[e], s[e], levels) << (BITS * e);
+            cw[i] = w;
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kBatch; ++i) {
+        if (BITS == 8)
+          *reinterpret_cast<uint32_t*>(out + i * row_stride) = cw[i];
+        else
+          *reinterpret_cast<uint16_t*>(out + i * row_stride) = (uint16_t)cw[i];
+      }
+    }
+  };
+  using std::integral_constant;
+  const bool rot = jb.unrotate_from >= 0;
+  if (bits == 8) {
+    if (rot) keys(integral_constant<int, 8>{}, integral_constant<bool, true>{});
+    else keys(integral_constant<int, 8>{}, integral_constant<bool, false>{});
+  } else {
+    if (rot) keys(integral_constant<int, 4>{}, integral_constant<bool, true>{});
+    else keys(integral_constant<int, 4>{}, integral_constant<bool, false>{});
   }
 }
 
-size_t quantize_smem() { return (size_t)kTokens * 2 * kD * 2 + (size_t)kTokens * 2 * kD; }  // tile + int8 code tile, 2 heads
+size_t quantize_smem(int hp) { return (size_t)kTokens * hp * kD * 2; }  // the 16-bit tile
+
+template <int DT, int HP>
+cudaError_t configure_one() {
+  return cudaFuncSetAttribute(quantize_batch_kernel<DT, HP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem(HP));
+}
 
 }  // namespace
 
 cudaError_t quantize_configure() {
-  cudaError_t e = cudaFuncSetAttribute(quantize_batch_kernel<KVB_DT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem());
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(quantize_batch_kernel<KVB_DT_F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)quantize_smem());
+  cudaError_t e = configure_one<KVB_DT_BF16, 1>();
+  if (e == cudaSuccess) e = configure_one<KVB_DT_BF16, 2>();
+  if (e == cudaSuccess) e = configure_one<KVB_DT_F16, 1>();
+  if (e == cudaSuccess) e = configure_one<KVB_DT_F16, 2>();
+  return e;
 }
 
 cudaError_t launch_quantize_batch(const QuantJob* jobs, int n_jobs, const ModelDims& m, const double* inv_freq, uint32_t* status,
                                   cudaStream_t st) {
-  const int n_hp = m.Hkv < 2 ? 1 : m.Hkv / 2;
-  const unsigned grid = (unsigned)n_jobs * m.L * 2 * n_hp;
-  if (m.dtype == KVB_DT_BF16)
-    quantize_batch_kernel<KVB_DT_BF16><<<grid, kThreads, quantize_smem(), st>>>(jobs, m, inv_freq, status);
-  else
-    quantize_batch_kernel<KVB_DT_F16><<<grid, kThreads, quantize_smem(), st>>>(jobs, m, inv_freq, status);
+  const int hp = m.Hkv < 2 ? 1 : 2;
+  const unsigned grid = (unsigned)n_jobs * m.L * 2 * (m.Hkv / hp);
+  const bool bf16 = m.dtype == KVB_DT_BF16;
+  if (hp == 2) {
+    if (bf16) quantize_batch_kernel<KVB_DT_BF16, 2><<<grid, kThreads, quantize_smem(2), st>>>(jobs, m, inv_freq, status);
+    else quantize_batch_kernel<KVB_DT_F16, 2><<<grid, kThreads, quantize_smem(2), st>>>(jobs, m, inv_freq, status);
+  } else {
+    if (bf16) quantize_batch_kernel<KVB_DT_BF16, 1><<<grid, kThreads, quantize_smem(1), st>>>(jobs, m, inv_freq, status);
+    else quantize_batch_kernel<KVB_DT_F16, 1><<<grid, kThreads, quantize_smem(1), st>>>(jobs, m, inv_freq, status);
+  }
   return cudaGetLastError();
 }
 
