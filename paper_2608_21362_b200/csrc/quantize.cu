@@ -191,6 +191,19 @@ __device__ __forceinline__ void store_meta(float* meta, size_t pair, float s, fl
   }
 }
 
+// (scale, min) as stored: what the second pass reads back for the values near a tie
+__device__ __forceinline__ void load_meta(const float* meta, size_t pair, int meta16, float& s, float& mn) {
+  if (meta16) {
+    const float2 t = __half22float2(reinterpret_cast<const __half2*>(meta)[pair]);
+    s = t.x, mn = t.y;
+  } else {
+    const float2 t = *reinterpret_cast<const float2*>(meta + pair * 2);
+    s = t.x, mn = t.y;
+  }
+}
+
+constexpr int kListCap = 2048;  // deferred items of a CTA (16 bits each)
+
 template <int DT, int HP>  // HP: KV heads of a CTA's tile (1 or 2)
 __global__ void __launch_bounds__(kThreads, 3)
     quantize_batch_kernel(const QuantJob* __restrict__ jobs, ModelDims m, const double* __restrict__ inv_freq,
@@ -200,8 +213,13 @@ __global__ void __launch_bounds__(kThreads, 3)
   constexpr int kParts = kThreads / NQ; // keys: parts of the tokens (4 or 8)
   constexpr int kTokPer = kTokens / kParts;  // keys: tokens of a part (32 or 16)
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) uint64_t bar;
-  __shared__ float4 s_mn[kThreads], s_mx[kThreads];  // keys: extremes of every (part, quad)
+  __shared__ __align__(8) uint64_t bar[4];  // one per quarter of the tokens: work starts when the first has landed
+  // keys: extremes of every (part, quad) while the parts of a group exchange them; afterwards, and for
+  // values from the start, s_mn holds the list of deferred items and s_mx the rotation coefficients of every quad
+  __shared__ float4 s_mn[kThreads], s_mx[kThreads];
+  __shared__ uint32_t s_n;                  // deferred items so far
+  uint16_t* s_list = reinterpret_cast<uint16_t*>(s_mn);  // kListCap items
+  static_assert(kListCap * sizeof(uint16_t) <= sizeof(float4) * kThreads, "the list overlays s_mn");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = m.Hkv;
   const int n_hp = H / HP;
@@ -221,29 +239,51 @@ __global__ void __launch_bounds__(kThreads, 3)
   const size_t layer_elems = (size_t)kTokens * E;
 
   // ------------------------------ the tile [128 tokens][HP heads][128 channels] into shared memory,
-  //                                all of it in flight at once
+  //                                all of it in flight at once, a barrier per 32 tokens
   constexpr uint32_t row_bytes = (uint32_t)W * 2;  // one token row of the tile
   uint16_t* s_x = reinterpret_cast<uint16_t*>(smem);  // [128][W]
   const uint16_t* tile = x + (size_t)l * layer_elems + (size_t)hb * kD;
   if (tid == 0) {
-    mbar_init(&bar, 1);
+    for (int q = 0; q < 4; ++q) mbar_init(&bar[q], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_n = 0;
   }
   __syncthreads();
   if (warp == 0) {
-    if (lane == 0) mbar_expect_tx(&bar, (uint32_t)kTokens * row_bytes);
+    if (lane < 4) mbar_expect_tx(&bar[lane], (uint32_t)(kTokens / 4) * row_bytes);
     __syncwarp();
     if (W == E) {  // the tile is one contiguous block -- four large copies
-      if (lane < 4) bulk_g2s(s_x + (size_t)lane * (kTokens / 4) * W, tile + (size_t)lane * (kTokens / 4) * W, (uint32_t)(kTokens / 4) * row_bytes, &bar);
+      if (lane < 4) bulk_g2s(s_x + (size_t)lane * (kTokens / 4) * W, tile + (size_t)lane * (kTokens / 4) * W, (uint32_t)(kTokens / 4) * row_bytes, &bar[lane]);
     } else {       // more heads: one copy per token row (the copy engine's request rate, not its bandwidth, sets the pace)
-      for (int t = lane; t < kTokens; t += 32) bulk_g2s(s_x + (size_t)t * W, tile + (size_t)t * E, row_bytes, &bar);
+      for (int t = lane; t < kTokens; t += 32) bulk_g2s(s_x + (size_t)t * W, tile + (size_t)t * E, row_bytes, &bar[t / (kTokens / 4)]);
     }
   }
-  const bool ok = __syncthreads_and(mbar_wait(&bar, 0));  // one answer for the whole CTA
-  if (!ok) {
-    if (tid == 0) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
-    return;
-  }
+  // Bounded wait for a quarter of the tokens.  A wait that gives up (never expected) reports it and lets the
+  // thread carry on over whatever the tile holds, so that no later barrier of the CTA is left waiting.
+  auto wait_quarter = [&](int q) {
+    if (!mbar_wait(&bar[q], 0)) atomicOr(status, DEV_STATUS_WAIT_TIMEOUT);
+  };
+  // Deferred items.  With 16-bit inputs the quotients of a group lie on a coarse lattice, so that about one
+  // value in 250 sits on or next to a tie; taking the IEEE division at once would leave nearly every warp
+  // running it with one or two lanes.  Instead the first pass stores the fast codes for everything and notes
+  // the places in a bit mask; the threads then put their places on a list of the CTA, and a second pass
+  // redoes the listed ones with the IEEE division, one item per thread (a thread whose places
+  // found no room on the list redoes them itself).
+  auto defer = [&](uint32_t mask, auto&& encode) -> uint32_t {  // returns the places that found no room
+    const int n = __popc(mask);
+    if (n == 0) return 0;
+    uint32_t pos = atomicAdd(&s_n, (uint32_t)n);
+    while (mask && pos < (uint32_t)kListCap) {
+      s_list[pos++] = (uint16_t)encode(__ffs(mask) - 1);
+      mask &= mask - 1;
+    }
+    return mask;
+  };
+  auto second_pass = [&](uint32_t left, auto&& encode, auto&& fix) {  // after a __syncthreads()
+    const int n = min(s_n, (uint32_t)kListCap);
+    for (int i = tid; i < n; i += kThreads) fix((uint32_t)s_list[i]);
+    for (; left; left &= left - 1) fix(encode(__ffs(left) - 1));
+  };
 
   if (kv) {
     // ------------------------------ values: eight lanes per (token, head) row, a warp takes four rows at
@@ -253,8 +293,27 @@ __global__ void __launch_bounds__(kThreads, 3)
     auto values = [&](auto bits_tag) {
       constexpr int BITS = decltype(bits_tag)::value;
       constexpr int G = BITS == 8 ? 1 : kD / 32;  // groups of a row: the whole row, or 32 channels each
+      constexpr int kPieces = G == 1 ? 1 : 2;     // groups a lane takes part in
+      constexpr int kLanes = G == 1 ? 8 : 4;      // lanes of a group
       const int sub = lane >> 3, lj = lane & 7;
-      for (int r = warp * 4 + sub; r < kTokens * HP; r += (kThreads / 32) * 4) {
+      // item: row | piece << 8 | lane of the row << 9 | word of the piece << 12 -- two values, two codes
+      auto fix = [&](uint32_t it) {
+        const int r = it & 255, p = (it >> 8) & 1, jj = (it >> 9) & 7, i = (it >> 12) & 3;
+        const size_t u = ((size_t)l * kTokens + r / HP) * H + hb + r % HP;
+        float s, mn, a, b;
+        load_meta(meta, u * G + (G == 1 ? 0 : 2 * p + (jj >> 2)), jb.meta16, s, mn);
+        f2_unpack(unpack2<DT>(*reinterpret_cast<const uint32_t*>(s_x + (size_t)r * kD + 64 * p + 8 * jj + 2 * i)), a, b);
+        const uint32_t c0 = code_exact(a, mn, s, levels), c1 = code_exact(b, mn, s, levels);
+        if (BITS == 8)
+          *reinterpret_cast<uint16_t*>(codes + u * kD + 64 * p + 8 * jj + 2 * i) = (uint16_t)(c0 | (c1 << 8));
+        else
+          codes[u * (kD / 2) + 32 * p + 4 * jj + i] = (uint8_t)(c0 | (c1 << 4));
+      };
+      uint32_t near_tie[2] = {0, 0};  // per piece: bit 4 * sweep + word
+#pragma unroll 2
+      for (int it = 0; it < 4 * HP; ++it) {  // 32 rows, i.e. 32 / HP tokens, per sweep of the CTA
+        if (it % HP == 0) wait_quarter(it / HP);
+        const int r = it * 32 + warp * 4 + sub;
         const int t = r / HP, hh = r % HP;
         const size_t u = ((size_t)l * kTokens + t) * H + hb + hh;  // (layer, token, head) row
         const uint4 wa = *reinterpret_cast<const uint4*>(s_x + (size_t)r * kD + 8 * lj);
@@ -270,9 +329,7 @@ __global__ void __launch_bounds__(kThreads, 3)
           lo[0] = min2_16<DT>(lo[0], lo[1]);
           hi[0] = max2_16<DT>(hi[0], hi[1]);
         }
-        constexpr int kPieces = G == 1 ? 1 : 2;     // groups this lane takes part in
-        constexpr int kLanes = G == 1 ? 8 : 4;      // lanes of a group
-        float mn[2], s[2], limit[2];
+        float limit[2];
         uint64_t mn2[2], inv2[2];
 #pragma unroll
         for (int p = 0; p < kPieces; ++p) {
@@ -281,55 +338,42 @@ __global__ void __launch_bounds__(kThreads, 3)
             lo[p] = min2_16<DT>(lo[p], __shfl_xor_sync(0xffffffffu, lo[p], o));
             hi[p] = max2_16<DT>(hi[p], __shfl_xor_sync(0xffffffffu, hi[p], o));
           }
-          float a, b, c, d;
+          float a, b, c, d, s;
           f2_unpack(unpack2<DT>(lo[p]), a, b);
           f2_unpack(unpack2<DT>(hi[p]), c, d);
-          mn[p] = fminf(a, b);
-          group_params(mn[p], fmaxf(c, d), levels, jb.meta16, s[p]);
+          float mn = fminf(a, b);
+          group_params(mn, fmaxf(c, d), levels, jb.meta16, s);
           const int g = G == 1 ? 0 : 2 * p + (lj >> 2);  // channels 8 lj (+ 64) lie in group lj / 4 (+ 2)
-          if ((lj & (kLanes - 1)) == 0) store_meta(meta, u * G + g, s[p], mn[p], jb.meta16);
-          const float inv = rcp_approx(s[p]);
-          mn2[p] = f2_pack(mn[p], mn[p]);
+          if ((lj & (kLanes - 1)) == 0) store_meta(meta, u * G + g, s, mn, jb.meta16);
+          const float inv = rcp_approx(s);
+          mn2[p] = f2_pack(mn, mn);
           inv2[p] = f2_pack(inv, inv);
-          limit[p] = trust_limit(s[p], levels);
+          limit[p] = trust_limit(s, levels);
         }
 #pragma unroll
         for (int p = 0; p < 2; ++p) {
           const int pp = G == 1 ? 0 : p;
-          float mq[4][2], rq[4][2], dev[4];
+          float mq[4][2], rq[4][2];
 #pragma unroll
-          for (int i = 0; i < 4; ++i) dev[i] = code_fast2(unpack2<DT>(w[p][i]), mn2[pp], inv2[pp], mq[i][0], mq[i][1], rq[i][0], rq[i][1]);
-          uint32_t out[2];
+          for (int i = 0; i < 4; ++i) {
+            const float dev = code_fast2(unpack2<DT>(w[p][i]), mn2[pp], inv2[pp], mq[i][0], mq[i][1], rq[i][0], rq[i][1]);
+            if (dev > limit[pp]) near_tie[p] |= 1u << (4 * it + i);
+          }
           if (BITS == 8) {
-            out[0] = pack4_u8(mq[0][0], mq[0][1], mq[1][0], mq[1][1]);
-            out[1] = pack4_u8(mq[2][0], mq[2][1], mq[3][0], mq[3][1]);
+            *reinterpret_cast<uint2*>(codes + u * kD + 64 * p + 8 * lj) =
+                make_uint2(pack4_u8(mq[0][0], mq[0][1], mq[1][0], mq[1][1]), pack4_u8(mq[2][0], mq[2][1], mq[3][0], mq[3][1]));
           } else {
-            out[0] = pack4_u8(pack2_u4(mq[0][0], rq[0][1]), pack2_u4(mq[1][0], rq[1][1]), pack2_u4(mq[2][0], rq[2][1]),
-                              pack2_u4(mq[3][0], rq[3][1]));
+            *reinterpret_cast<uint32_t*>(codes + u * (kD / 2) + 32 * p + 4 * lj) =
+                pack4_u8(pack2_u4(mq[0][0], rq[0][1]), pack2_u4(mq[1][0], rq[1][1]), pack2_u4(mq[2][0], rq[2][1]), pack2_u4(mq[3][0], rq[3][1]));
           }
-          const float worst = fmaxf(fmaxf(dev[0], dev[1]), fmaxf(dev[2], dev[3]));
-          if (__any_sync(0xffffffffu, worst > limit[pp])) {  // rare: the IEEE division decides for the words near a tie
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              if (dev[i] > limit[pp]) {
-                float a, b;
-                f2_unpack(unpack2<DT>(w[p][i]), a, b);
-                const uint32_t c0 = code_exact(a, mn[pp], s[pp], levels), c1 = code_exact(b, mn[pp], s[pp], levels);
-                if (BITS == 8) {
-                  const int sh = (i & 1) * 16;
-                  out[i >> 1] = (out[i >> 1] & ~(0xFFFFu << sh)) | ((c0 | (c1 << 8)) << sh);
-                } else {
-                  out[0] = (out[0] & ~(0xFFu << (8 * i))) | ((c0 | (c1 << 4)) << (8 * i));
-                }
-              }
-            }
-          }
-          if (BITS == 8)
-            *reinterpret_cast<uint2*>(codes + u * kD + 64 * p + 8 * lj) = make_uint2(out[0], out[1]);
-          else
-            *reinterpret_cast<uint32_t*>(codes + u * (kD / 2) + 32 * p + 4 * lj) = out[0];
         }
       }
+      auto place0 = [&](int b) { return (uint32_t)((b >> 2) * 32 + warp * 4 + sub) | (lj << 9) | ((b & 3) << 12); };
+      auto place1 = [&](int b) { return place0(b) | (1u << 8); };
+      const uint32_t left0 = defer(near_tie[0], place0), left1 = defer(near_tie[1], place1);
+      __syncthreads();
+      second_pass(left0, place0, fix);
+      for (uint32_t left = left1; left; left &= left - 1) fix(place1(__ffs(left) - 1));
     };
     if (bits == 8) values(std::integral_constant<int, 8>{});
     else values(std::integral_constant<int, 4>{});
@@ -342,9 +386,7 @@ __global__ void __launch_bounds__(kThreads, 3)
   // run as packed float32 pairs, and a token's four codes leave with one store.
   const int quad = tid % NQ;                 // tile channels 4 quad .. 4 quad + 3
   const int part = tid / NQ;                 // tokens part * kTokPer .. + kTokPer - 1
-  const int c = 4 * quad;
-  const int h = hb + c / kD, j = c % kD;
-  const uint2* s_q = reinterpret_cast<const uint2*>(s_x);  // [128][NQ] words pairs of four channels
+  const uint2* s_q = reinterpret_cast<const uint2*>(s_x);  // [128][NQ] word pairs of four channels
 
   auto keys = [&](auto bits_tag, auto rot_tag) {
     constexpr int BITS = decltype(bits_tag)::value;
@@ -352,8 +394,12 @@ __global__ void __launch_bounds__(kThreads, 3)
     constexpr int kGroupTokens = BITS == 8 ? kTokens : 32;  // one group per chunk, or groups of 32 tokens
     constexpr int G = kTokens / kGroupTokens;
     constexpr int kPartsPerGroup = kGroupTokens / kTokPer;
-    uint64_t cs2[2] = {0, 0}, sn2[2] = {0, 0};
+    constexpr int kBatch = 4;
+    const size_t row_stride = (size_t)E * BITS / 8;  // bytes of a token row of the layer's codes
+    uint8_t* const out_tile = codes + (((size_t)l * layer_elems + (size_t)hb * kD) * BITS) / 8;
+    float4 cs4 = make_float4(0.f, 0.f, 0.f, 0.f), sn4 = cs4;
     if (ROT) {  // channel j pairs with j + 64: low half + x_hi * s, high half - x_lo * s
+      const int j = (4 * quad) % kD;
       float cs[4], sn[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -362,21 +408,45 @@ __global__ void __launch_bounds__(kThreads, 3)
         cs[i] = (float)c_d;
         sn[i] = j < 64 ? (float)s_d : -(float)s_d;
       }
-      cs2[0] = f2_pack(cs[0], cs[1]), cs2[1] = f2_pack(cs[2], cs[3]);
-      sn2[0] = f2_pack(sn[0], sn[1]), sn2[1] = f2_pack(sn[2], sn[3]);
+      cs4 = make_float4(cs[0], cs[1], cs[2], cs[3]);
+      sn4 = make_float4(sn[0], sn[1], sn[2], sn[3]);
     }
-    // the four values of token t as two packed pairs
-    auto value4 = [&](int t, uint64_t& v01, uint64_t& v23) {
-      const uint2 w = s_q[t * NQ + quad];
+    // the four values of token t, quad qd, as two packed pairs (c, s: the quad's rotation coefficients)
+    auto value4 = [&](int t, int qd, const float4& c, const float4& s, uint64_t& v01, uint64_t& v23) {
+      const uint2 w = s_q[t * NQ + qd];
       v01 = unpack2<DT>(w.x), v23 = unpack2<DT>(w.y);
       if (ROT) {  // per value: fma(x, c, x_partner * s), as the one-chunk form
-        const uint2 wp = s_q[t * NQ + (quad ^ 16)];
-        v01 = f2_fma(v01, cs2[0], f2_mul(unpack2<DT>(wp.x), sn2[0]));
-        v23 = f2_fma(v23, cs2[1], f2_mul(unpack2<DT>(wp.y), sn2[1]));
+        const uint2 wp = s_q[t * NQ + (qd ^ 16)];
+        v01 = f2_fma(v01, f2_pack(c.x, c.y), f2_mul(unpack2<DT>(wp.x), f2_pack(s.x, s.y)));
+        v23 = f2_fma(v23, f2_pack(c.z, c.w), f2_mul(unpack2<DT>(wp.y), f2_pack(s.z, s.w)));
       }
+    };
+    // item: token | quad << 7 -- the token's four codes of that quad, redone with the IEEE division against
+    // the (scale, min) the group stored
+    auto fix = [&](uint32_t it) {
+      const int t = it & 127, qd = it >> 7;
+      const int h = hb + (4 * qd) / kD, j = (4 * qd) % kD;
+      const size_t pair = (((size_t)l * G + t / kGroupTokens) * H + h) * kD + j;
+      uint64_t v01, v23;
+      if (ROT) value4(t, qd, s_mx[qd], s_mx[NQ + qd], v01, v23);
+      else value4(t, qd, cs4, sn4, v01, v23);
+      float v[4];
+      f2_unpack(v01, v[0], v[1]);
+      f2_unpack(v23, v[2], v[3]);
+      uint32_t w = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        float s, mn;
+        load_meta(meta, pair + e, jb.meta16, s, mn);
+        w |= code_exact(v[e], mn, s, levels) << (BITS * e);
+      }
+      uint8_t* o = out_tile + (size_t)t * row_stride + (4 * qd * BITS) / 8;
+      if (BITS == 8) *reinterpret_cast<uint32_t*>(o) = w;
+      else *reinterpret_cast<uint16_t*>(o) = (uint16_t)w;
     };
     // ---- extremes of this part's tokens
     const int t0 = part * kTokPer;
+    wait_quarter(t0 / (kTokens / 4));
     float mn[4], mx[4];
     if (!ROT) {
       uint2 lo = s_q[t0 * NQ + quad], hi = lo;
@@ -396,7 +466,7 @@ __global__ void __launch_bounds__(kThreads, 3)
 #pragma unroll 4
       for (int t = t0; t < t0 + kTokPer; ++t) {
         uint64_t v01, v23;
-        value4(t, v01, v23);
+        value4(t, quad, cs4, sn4, v01, v23);
         float v[4];
         f2_unpack(v01, v[0], v[1]);
         f2_unpack(v23, v[2], v[3]);
@@ -422,46 +492,29 @@ __global__ void __launch_bounds__(kThreads, 3)
       limit = fminf(limit, trust_limit(s[i], levels));
     }
     if (part % kPartsPerGroup == 0) {
-      const size_t pair = (((size_t)l * G + g) * H + h) * kD + j;
+      const size_t pair = (((size_t)l * G + g) * H + hb + (4 * quad) / kD) * kD + (4 * quad) % kD;
 #pragma unroll
       for (int i = 0; i < 4; ++i) store_meta(meta, pair + i, s[i], mn[i], jb.meta16);
     }
-    // ---- codes, kBatch tokens at a time
-    constexpr int kBatch = 4;
+    // ---- first pass: the fast codes of every token, kBatch tokens at a time; a bit per token near a tie
     const uint64_t mn01 = f2_pack(mn[0], mn[1]), mn23 = f2_pack(mn[2], mn[3]);
     const uint64_t inv01 = f2_pack(rcp_approx(s[0]), rcp_approx(s[1])), inv23 = f2_pack(rcp_approx(s[2]), rcp_approx(s[3]));
-    const size_t row_stride = (size_t)E * BITS / 8;  // bytes of a token row of the layer's codes
-    uint8_t* out = codes + (((size_t)l * layer_elems + (size_t)hb * kD + c) * BITS) / 8 + (size_t)t0 * row_stride;
-    for (int t8 = t0; t8 < t0 + kTokPer; t8 += kBatch, out += kBatch * row_stride) {
+    uint8_t* out = out_tile + (size_t)t0 * row_stride + (4 * quad * BITS) / 8;
+    uint32_t near_tie = 0;  // bit t - t0
+#pragma unroll 1
+    for (int tb = 0; tb < kTokPer; tb += kBatch, out += kBatch * row_stride) {
       uint32_t cw[kBatch];
-      float dev[kBatch], worst = 0.f;
 #pragma unroll
       for (int i = 0; i < kBatch; ++i) {
         uint64_t v01, v23;
-        value4(t8 + i, v01, v23);
+        value4(t0 + tb + i, quad, cs4, sn4, v01, v23);
         float ma[2], mb[2], ra[2], rb[2];
-        dev[i] = fmaxf(code_fast2(v01, mn01, inv01, ma[0], ma[1], ra[0], ra[1]), code_fast2(v23, mn23, inv23, mb[0], mb[1], rb[0], rb[1]));
-        worst = fmaxf(worst, dev[i]);
+        const float dev = fmaxf(code_fast2(v01, mn01, inv01, ma[0], ma[1], ra[0], ra[1]), code_fast2(v23, mn23, inv23, mb[0], mb[1], rb[0], rb[1]));
+        if (dev > limit) near_tie |= 1u << (tb + i);
         if (BITS == 8)
           cw[i] = pack4_u8(ma[0], ma[1], mb[0], mb[1]);
         else
           cw[i] = __float_as_uint(fmaf(pack2_u4(rb[0], rb[1]), 256.f, pack2_u4(ma[0], ra[1])));  // low 16 bits
-      }
-      if (__any_sync(0xffffffffu, worst > limit)) {  // rare: the IEEE division decides for the tokens near a tie
-#pragma unroll
-        for (int i = 0; i < kBatch; ++i) {
-          if (dev[i] > limit) {
-            uint64_t v01, v23;
-            value4(t8 + i, v01, v23);
-            float v[4];
-            f2_unpack(v01, v[0], v[1]);
-            f2_unpack(v23, v[2], v[3]);
-            uint32_t w = 0;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) w |= code_exact(v[e], mn[e], s[e], levels) << (BITS * e);
-            cw[i] = w;
-          }
-        }
       }
 #pragma unroll
       for (int i = 0; i < kBatch; ++i) {
@@ -471,6 +524,13 @@ __global__ void __launch_bounds__(kThreads, 3)
           *reinterpret_cast<uint16_t*>(out + i * row_stride) = (uint16_t)cw[i];
       }
     }
+    // ---- second pass.  The exchange arrays are free once every thread has read them.
+    __syncthreads();
+    if (ROT && part == 0) s_mx[quad] = cs4, s_mx[NQ + quad] = sn4;
+    auto place = [&](int b) { return (uint32_t)(t0 + b) | ((uint32_t)quad << 7); };
+    const uint32_t left = defer(near_tie, place);
+    __syncthreads();
+    second_pass(left, place, fix);
   };
   using std::integral_constant;
   const bool rot = jb.unrotate_from >= 0;

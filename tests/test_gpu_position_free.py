@@ -116,6 +116,7 @@ def test_batched_quantiser_codes_bit_exact(kv_dtype, Hkv):
         specs = [  # (bits, keys?, values?, unrotate_from, meta_fp16)
             (8, True, True, -1, False), (4, True, True, -1, False), (8, True, False, 4096 + 128, False), (4, True, True, 77, False),
             (8, False, True, -1, False), (4, True, True, -1, True), (8, True, True, (1 << 24) - 128, True), (8, True, True, -1, False),
+            (8, True, True, -1, False), (4, True, True, -1, True),  # 8, 9: every other quotient an exact tie (below)
         ]
         jobs, xs = [], []
         for i, (bits, has_k, has_v, pos, m16) in enumerate(specs):
@@ -127,6 +128,15 @@ def test_batched_quantiser_codes_bit_exact(kv_dtype, Hkv):
                 k[:, :, :, 9] = 1.0
                 k[:, 64:, :, 9] = 1.0 + 2.0 ** -7
                 v[:, 7, :, ::2] = 3.0e4 if kv_dtype == "fp16" else 1.0e30
+            if i >= 8:  # integers in [0, 2 * levels] with both ends in every group: scale 2, the odd ones tie, far
+                # more of them than the kernel's list of places to redo with the IEEE division holds
+                top = 2 * ((1 << bits) - 1)
+                g = torch.Generator().manual_seed(300 + i)
+                k = torch.randint(0, top // 2 + 1, (sh.L, sh.C, Hkv, sh.d), generator=g).float()
+                v = torch.randint(0, top // 2 + 1, (sh.L, sh.C, Hkv, sh.d), generator=g).float()
+                k[:, 0::32], k[:, 1::32] = 0.0, float(top)              # keys: groups run over tokens
+                v[:, :, :, 0::32], v[:, :, :, 1::32] = 0.0, float(top)  # values: over channels
+                k, v = k.to(sh.torch_dtype), v.to(sh.torch_dtype)
             mt = torch.float16 if m16 else torch.float32
             j = dict(bits=bits, unrotate_from=pos, meta_fp16=m16)
             if has_k:
