@@ -3,23 +3,25 @@
 // scale = (max-min)/(2^b-1) and min are float32; the code is rint((x-min)/scale) in float32
 // (IEEE subtract, divide, round-half-even), clamped.  A constant group gets scale 1, codes 0.
 //
-// One launch quantises a batch of chunks: a CTA per (chunk, layer, K|V, pair of KV heads).
-//   keys    the CTA's [128 tokens][<= 2 heads][128 channels] tile is fetched into shared memory by
-//           bulk copies (four large ones where the tile is contiguous, i.e. up to two KV heads;
-//           one per token row otherwise); a thread owns a PAIR of neighbouring channels and a
-//           part of the tokens (one four-byte load per token brings both values, the arithmetic
-//           runs on packed float32 pairs), walks its token groups twice (extremes, then codes;
-//           with one group per chunk the parts exchange their extremes through shared memory)
-//           and leaves the codes in a shared-memory tile that the CTA writes out in 16-byte
-//           pieces.  With `unrotate` every key is first rotated back
-//           by R_theta^(-orig_pos) (Rotary Positional Embeddings, Eq. 3), so that the stored
-//           chunk is position-free and re-use at new_pos needs the single rotation by new_pos;
-//           cos / sin come from a double-precision angle, the rotation itself is float32 in a
-//           fixed order: u = fma(x, c, +-(x_partner * s)).
-//   values  the same tile, staged the same way; a warp per (token, head) row, 4 channels per lane.
-// The division of the code decision is the hardware reciprocal where that provably gives the
-// same integer (the quotient lies away from every half-integer) and the IEEE division otherwise,
-// decided per warp and batch of eight tokens so that the common case carries no division at all.
+// One launch quantises a batch of chunks: a CTA per (chunk, layer, K|V, pair of KV heads), three CTAs per SM.
+// The CTA's [128 tokens][<= 2 heads][128 channels] tile is fetched into shared memory by bulk copies
+// (four large ones where the tile is contiguous, i.e. up to two KV heads; one per token row
+// otherwise), with a barrier per 32 tokens so that work starts when the first quarter has landed.
+//   keys    a thread owns a QUAD of neighbouring channels and a part of the tokens: one eight-byte load
+//           per token brings the four values; the extremes are taken on the 16-bit values, two per
+//           instruction; the parts of a group exchange their extremes through shared memory; the
+//           codes come from packed float32 pairs and leave with one store per token.  With `unrotate`
+//           every key is first rotated back by R_theta^(-orig_pos) (Rotary Positional Embeddings,
+//           Eq. 3), so that the stored chunk is position-free and re-use at new_pos needs the single
+//           rotation by new_pos; cos / sin come from a double-precision angle, the rotation itself
+//           is float32 in a fixed order: u = fma(x, c, +-(x_partner * s)).
+//   values  eight lanes per (token, head) row, 16 channels per lane, the extremes reduced by shuffles
+//           of packed 16-bit words.
+// The division of the code decision is the hardware reciprocal where that provably gives the same
+// integer (the quotient lies away from every half-integer).  The other values -- with 16-bit inputs the
+// quotients of a group lie on a coarse lattice, so about one in 250 is a tie or next to one -- are
+// marked in a bit mask, collected on a list of the CTA and redone with the IEEE division in a second
+// pass, one item per thread, so that neither pass runs with a few lanes of a warp.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -130,8 +132,14 @@ __device__ __forceinline__ float rcp_approx(float x) {
   return y;
 }
 __device__ __forceinline__ bool scale_usable(float s) { return s >= 1e-30f && s <= 1e30f; }
-// largest |q - rint(q)| for which the fast code is trusted; below zero when the scale is not usable
-__device__ __forceinline__ float trust_limit(float s, float levels) { return scale_usable(s) ? 0.5f - 4e-7f * levels : -1.f; }
+// Largest |q - rint(q)| for which the fast code is trusted, as the bit pattern of that float (for
+// non-negative floats the integer order of the patterns is the order of the values); -1, below every
+// pattern, when the scale is not usable.
+__device__ __forceinline__ int32_t trust_limit(float s, float levels) { return scale_usable(s) ? __float_as_int(0.5f - 4e-7f * levels) : -1; }
+// shifts `marks` left by one and brings in a 1 when dev > limit (dev >= 0): the sign of limit - dev
+__device__ __forceinline__ uint32_t mark_near_tie(uint32_t marks, float dev, int32_t limit) {
+  return __funnelshift_l((uint32_t)(limit - __float_as_int(dev)), marks, 1);
+}
 
 // four codes, each in the low byte of m_i's bit pattern, as one word (code 0 in the lowest byte)
 __device__ __forceinline__ uint32_t pack4_u8(float m0, float m1, float m2, float m3) {
@@ -183,7 +191,7 @@ __device__ __forceinline__ void group_params(float& mn, float mx, float levels, 
   s = mx > mn ? __fdiv_rn(__fsub_rn(mx, mn), levels) : 1.0f;
   if (meta16) s = __half2float(__float2half_ru(s));
 }
-__device__ __forceinline__ void store_meta(float* meta, size_t pair, float s, float mn, int meta16) {
+__device__ __forceinline__ void store_meta(float* meta, uint32_t pair, float s, float mn, int meta16) {
   if (meta16) {
     reinterpret_cast<__half2*>(meta)[pair] = __floats2half2_rn(s, mn);  // both already binary16 values
   } else {
@@ -192,7 +200,7 @@ __device__ __forceinline__ void store_meta(float* meta, size_t pair, float s, fl
 }
 
 // (scale, min) as stored: what the second pass reads back for the values near a tie
-__device__ __forceinline__ void load_meta(const float* meta, size_t pair, int meta16, float& s, float& mn) {
+__device__ __forceinline__ void load_meta(const float* meta, uint32_t pair, int meta16, float& s, float& mn) {
   if (meta16) {
     const float2 t = __half22float2(reinterpret_cast<const __half2*>(meta)[pair]);
     s = t.x, mn = t.y;
@@ -200,6 +208,11 @@ __device__ __forceinline__ void load_meta(const float* meta, size_t pair, int me
     const float2 t = *reinterpret_cast<const float2*>(meta + pair * 2);
     s = t.x, mn = t.y;
   }
+}
+
+// the metadata of pair number `pairs` onward
+__device__ __forceinline__ float* meta_from(float* meta, size_t pairs, int meta16) {
+  return reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(meta) + pairs * (meta16 ? 4 : 8));
 }
 
 constexpr int kListCap = 2048;  // deferred items of a CTA (16 bits each)
@@ -295,27 +308,31 @@ __global__ void __launch_bounds__(kThreads, 3)
       constexpr int G = BITS == 8 ? 1 : kD / 32;  // groups of a row: the whole row, or 32 channels each
       constexpr int kPieces = G == 1 ? 1 : 2;     // groups a lane takes part in
       constexpr int kLanes = G == 1 ? 8 : 4;      // lanes of a group
+      constexpr int kSweeps = 4 * HP;             // 32 rows, i.e. 32 / HP tokens, per sweep of the CTA
       const int sub = lane >> 3, lj = lane & 7;
+      // this layer's rows: row u = token * H + head, 32-bit offsets from here on
+      uint8_t* const codes_l = codes + (size_t)l * kTokens * H * (kD * BITS / 8);
+      float* const meta_l = meta_from(meta, (size_t)l * kTokens * H * G, jb.meta16);
       // item: row | piece << 8 | lane of the row << 9 | word of the piece << 12 -- two values, two codes
       auto fix = [&](uint32_t it) {
         const int r = it & 255, p = (it >> 8) & 1, jj = (it >> 9) & 7, i = (it >> 12) & 3;
-        const size_t u = ((size_t)l * kTokens + r / HP) * H + hb + r % HP;
+        const uint32_t u = (uint32_t)((r / HP) * H + hb + r % HP);
         float s, mn, a, b;
-        load_meta(meta, u * G + (G == 1 ? 0 : 2 * p + (jj >> 2)), jb.meta16, s, mn);
+        load_meta(meta_l, u * G + (G == 1 ? 0 : 2 * p + (jj >> 2)), jb.meta16, s, mn);
         f2_unpack(unpack2<DT>(*reinterpret_cast<const uint32_t*>(s_x + (size_t)r * kD + 64 * p + 8 * jj + 2 * i)), a, b);
         const uint32_t c0 = code_exact(a, mn, s, levels), c1 = code_exact(b, mn, s, levels);
         if (BITS == 8)
-          *reinterpret_cast<uint16_t*>(codes + u * kD + 64 * p + 8 * jj + 2 * i) = (uint16_t)(c0 | (c1 << 8));
+          *reinterpret_cast<uint16_t*>(codes_l + u * kD + 64 * p + 8 * jj + 2 * i) = (uint16_t)(c0 | (c1 << 8));
         else
-          codes[u * (kD / 2) + 32 * p + 4 * jj + i] = (uint8_t)(c0 | (c1 << 4));
+          codes_l[u * (kD / 2) + 32 * p + 4 * jj + i] = (uint8_t)(c0 | (c1 << 4));
       };
-      uint32_t near_tie[2] = {0, 0};  // per piece: bit 4 * sweep + word
+      uint32_t near_tie[2] = {0, 0};  // per piece: a bit per (sweep, word), the last one lowest
 #pragma unroll 2
-      for (int it = 0; it < 4 * HP; ++it) {  // 32 rows, i.e. 32 / HP tokens, per sweep of the CTA
+      for (int it = 0; it < kSweeps; ++it) {
         if (it % HP == 0) wait_quarter(it / HP);
         const int r = it * 32 + warp * 4 + sub;
         const int t = r / HP, hh = r % HP;
-        const size_t u = ((size_t)l * kTokens + t) * H + hb + hh;  // (layer, token, head) row
+        const uint32_t u = (uint32_t)(t * H + hb + hh);  // (token, head) row of the layer
         const uint4 wa = *reinterpret_cast<const uint4*>(s_x + (size_t)r * kD + 8 * lj);
         const uint4 wb = *reinterpret_cast<const uint4*>(s_x + (size_t)r * kD + 64 + 8 * lj);
         const uint32_t w[2][4] = {{wa.x, wa.y, wa.z, wa.w}, {wb.x, wb.y, wb.z, wb.w}};
@@ -329,7 +346,7 @@ __global__ void __launch_bounds__(kThreads, 3)
           lo[0] = min2_16<DT>(lo[0], lo[1]);
           hi[0] = max2_16<DT>(hi[0], hi[1]);
         }
-        float limit[2];
+        int32_t limit[2];
         uint64_t mn2[2], inv2[2];
 #pragma unroll
         for (int p = 0; p < kPieces; ++p) {
@@ -344,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, 3)
           float mn = fminf(a, b);
           group_params(mn, fmaxf(c, d), levels, jb.meta16, s);
           const int g = G == 1 ? 0 : 2 * p + (lj >> 2);  // channels 8 lj (+ 64) lie in group lj / 4 (+ 2)
-          if ((lj & (kLanes - 1)) == 0) store_meta(meta, u * G + g, s, mn, jb.meta16);
+          if ((lj & (kLanes - 1)) == 0) store_meta(meta_l, u * G + g, s, mn, jb.meta16);
           const float inv = rcp_approx(s);
           mn2[p] = f2_pack(mn, mn);
           inv2[p] = f2_pack(inv, inv);
@@ -357,18 +374,21 @@ __global__ void __launch_bounds__(kThreads, 3)
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const float dev = code_fast2(unpack2<DT>(w[p][i]), mn2[pp], inv2[pp], mq[i][0], mq[i][1], rq[i][0], rq[i][1]);
-            if (dev > limit[pp]) near_tie[p] |= 1u << (4 * it + i);
+            near_tie[p] = mark_near_tie(near_tie[p], dev, limit[pp]);
           }
           if (BITS == 8) {
-            *reinterpret_cast<uint2*>(codes + u * kD + 64 * p + 8 * lj) =
+            *reinterpret_cast<uint2*>(codes_l + u * kD + 64 * p + 8 * lj) =
                 make_uint2(pack4_u8(mq[0][0], mq[0][1], mq[1][0], mq[1][1]), pack4_u8(mq[2][0], mq[2][1], mq[3][0], mq[3][1]));
           } else {
-            *reinterpret_cast<uint32_t*>(codes + u * (kD / 2) + 32 * p + 4 * lj) =
+            *reinterpret_cast<uint32_t*>(codes_l + u * (kD / 2) + 32 * p + 4 * lj) =
                 pack4_u8(pack2_u4(mq[0][0], rq[0][1]), pack2_u4(mq[1][0], rq[1][1]), pack2_u4(mq[2][0], rq[2][1]), pack2_u4(mq[3][0], rq[3][1]));
           }
         }
       }
-      auto place0 = [&](int b) { return (uint32_t)((b >> 2) * 32 + warp * 4 + sub) | (lj << 9) | ((b & 3) << 12); };
+      auto place0 = [&](int b) {  // bit b: sweep and word number 4 * kSweeps - 1 - b
+        const int n = 4 * kSweeps - 1 - b;
+        return (uint32_t)((n >> 2) * 32 + warp * 4 + sub) | (lj << 9) | ((n & 3) << 12);
+      };
       auto place1 = [&](int b) { return place0(b) | (1u << 8); };
       const uint32_t left0 = defer(near_tie[0], place0), left1 = defer(near_tie[1], place1);
       __syncthreads();
@@ -395,8 +415,9 @@ __global__ void __launch_bounds__(kThreads, 3)
     constexpr int G = kTokens / kGroupTokens;
     constexpr int kPartsPerGroup = kGroupTokens / kTokPer;
     constexpr int kBatch = 4;
-    const size_t row_stride = (size_t)E * BITS / 8;  // bytes of a token row of the layer's codes
-    uint8_t* const out_tile = codes + (((size_t)l * layer_elems + (size_t)hb * kD) * BITS) / 8;
+    const uint32_t row_stride = (uint32_t)E * BITS / 8;  // bytes of a token row of the layer's codes
+    uint8_t* const out_tile = codes + (((size_t)l * layer_elems + (size_t)hb * kD) * BITS) / 8;  // 32-bit offsets from here on
+    float* const meta_l = meta_from(meta, (size_t)l * G * H * kD, jb.meta16);
     float4 cs4 = make_float4(0.f, 0.f, 0.f, 0.f), sn4 = cs4;
     if (ROT) {  // channel j pairs with j + 64: low half + x_hi * s, high half - x_lo * s
       const int j = (4 * quad) % kD;
@@ -426,7 +447,7 @@ __global__ void __launch_bounds__(kThreads, 3)
     auto fix = [&](uint32_t it) {
       const int t = it & 127, qd = it >> 7;
       const int h = hb + (4 * qd) / kD, j = (4 * qd) % kD;
-      const size_t pair = (((size_t)l * G + t / kGroupTokens) * H + h) * kD + j;
+      const uint32_t pair = (uint32_t)(((t / kGroupTokens) * H + h) * kD + j);
       uint64_t v01, v23;
       if (ROT) value4(t, qd, s_mx[qd], s_mx[NQ + qd], v01, v23);
       else value4(t, qd, cs4, sn4, v01, v23);
@@ -437,10 +458,10 @@ __global__ void __launch_bounds__(kThreads, 3)
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         float s, mn;
-        load_meta(meta, pair + e, jb.meta16, s, mn);
+        load_meta(meta_l, pair + e, jb.meta16, s, mn);
         w |= code_exact(v[e], mn, s, levels) << (BITS * e);
       }
-      uint8_t* o = out_tile + (size_t)t * row_stride + (4 * qd * BITS) / 8;
+      uint8_t* o = out_tile + (uint32_t)t * row_stride + (uint32_t)(4 * qd * BITS) / 8;
       if (BITS == 8) *reinterpret_cast<uint32_t*>(o) = w;
       else *reinterpret_cast<uint16_t*>(o) = (uint16_t)w;
     };
@@ -485,22 +506,23 @@ __global__ void __launch_bounds__(kThreads, 3)
       mn[0] = fminf(mn[0], a.x), mn[1] = fminf(mn[1], a.y), mn[2] = fminf(mn[2], a.z), mn[3] = fminf(mn[3], a.w);
       mx[0] = fmaxf(mx[0], b.x), mx[1] = fmaxf(mx[1], b.y), mx[2] = fmaxf(mx[2], b.z), mx[3] = fmaxf(mx[3], b.w);
     }
-    float s[4], limit = 1.f;
+    float s[4];
+    int32_t limit = 0x7fffffff;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       group_params(mn[i], mx[i], levels, jb.meta16, s[i]);
-      limit = fminf(limit, trust_limit(s[i], levels));
+      limit = min(limit, trust_limit(s[i], levels));
     }
     if (part % kPartsPerGroup == 0) {
-      const size_t pair = (((size_t)l * G + g) * H + hb + (4 * quad) / kD) * kD + (4 * quad) % kD;
+      const uint32_t pair = (uint32_t)((g * H + hb + (4 * quad) / kD) * kD + (4 * quad) % kD);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) store_meta(meta, pair + i, s[i], mn[i], jb.meta16);
+      for (int i = 0; i < 4; ++i) store_meta(meta_l, pair + i, s[i], mn[i], jb.meta16);
     }
     // ---- first pass: the fast codes of every token, kBatch tokens at a time; a bit per token near a tie
     const uint64_t mn01 = f2_pack(mn[0], mn[1]), mn23 = f2_pack(mn[2], mn[3]);
     const uint64_t inv01 = f2_pack(rcp_approx(s[0]), rcp_approx(s[1])), inv23 = f2_pack(rcp_approx(s[2]), rcp_approx(s[3]));
-    uint8_t* out = out_tile + (size_t)t0 * row_stride + (4 * quad * BITS) / 8;
-    uint32_t near_tie = 0;  // bit t - t0
+    uint32_t out = (uint32_t)t0 * row_stride + (uint32_t)(4 * quad * BITS) / 8;  // offset in out_tile
+    uint32_t near_tie = 0;  // a bit per token, the last one lowest
 #pragma unroll 1
     for (int tb = 0; tb < kTokPer; tb += kBatch, out += kBatch * row_stride) {
       uint32_t cw[kBatch];
@@ -510,7 +532,7 @@ __global__ void __launch_bounds__(kThreads, 3)
         value4(t0 + tb + i, quad, cs4, sn4, v01, v23);
         float ma[2], mb[2], ra[2], rb[2];
         const float dev = fmaxf(code_fast2(v01, mn01, inv01, ma[0], ma[1], ra[0], ra[1]), code_fast2(v23, mn23, inv23, mb[0], mb[1], rb[0], rb[1]));
-        if (dev > limit) near_tie |= 1u << (tb + i);
+        near_tie = mark_near_tie(near_tie, dev, limit);
         if (BITS == 8)
           cw[i] = pack4_u8(ma[0], ma[1], mb[0], mb[1]);
         else
@@ -519,15 +541,15 @@ __global__ void __launch_bounds__(kThreads, 3)
 #pragma unroll
       for (int i = 0; i < kBatch; ++i) {
         if (BITS == 8)
-          *reinterpret_cast<uint32_t*>(out + i * row_stride) = cw[i];
+          *reinterpret_cast<uint32_t*>(out_tile + (out + i * row_stride)) = cw[i];
         else
-          *reinterpret_cast<uint16_t*>(out + i * row_stride) = (uint16_t)cw[i];
+          *reinterpret_cast<uint16_t*>(out_tile + (out + i * row_stride)) = (uint16_t)cw[i];
       }
     }
     // ---- second pass.  The exchange arrays are free once every thread has read them.
     __syncthreads();
     if (ROT && part == 0) s_mx[quad] = cs4, s_mx[NQ + quad] = sn4;
-    auto place = [&](int b) { return (uint32_t)(t0 + b) | ((uint32_t)quad << 7); };
+    auto place = [&](int b) { return (uint32_t)(t0 + kTokPer - 1 - b) | ((uint32_t)quad << 7); };
     const uint32_t left = defer(near_tie, place);
     __syncthreads();
     second_pass(left, place, fix);
