@@ -643,31 +643,32 @@ int kvb_patch(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_selectio
   if (!sel) return fail(c, KVB_ERR_INVALID_ARG, "NULL selection array");
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   KVB_CUDA(c, cudaSetDevice(c->device));
-  uint8_t* host = nullptr;
-  const int slot_code = take_slot(c, &host);
-  if (slot_code >= 0) return slot_code;
-  const int slot = -slot_code - 1;
-  ReqDesc* rd = reinterpret_cast<ReqDesc*>(host);
-  const int rows_per_cta = 64;
-  int tiles = 0;
-  for (int r = 0; r < n_req; ++r) {
-    const kvb_selection& s = sel[r];
-    if (!s.sel || !s.n_sel || s.sel_capacity <= 0) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL sel / n_sel or empty capacity", r);
-    ReqDesc d{};
-    d.kv_buf = static_cast<const uint8_t*>(reqs[r].kv_buf);
-    d.fresh = static_cast<const uint8_t*>(reqs[r].fresh);
-    d.sel = s.sel;
-    d.n_sel = s.n_sel;
-    d.T = reqs[r].T;
-    d.sel_capacity = s.sel_capacity;
-    d.tile_offset = tiles;
-    rd[r] = d;
-    tiles += (s.sel_capacity + rows_per_cta - 1) / rows_per_cta;
+  auto fill = [&](PatchDesc* out) -> int {
+    for (int r = 0; r < n_req; ++r) {
+      const kvb_selection& s = sel[r];
+      if (!s.sel || !s.n_sel || s.sel_capacity <= 0) return fail(c, KVB_ERR_INVALID_ARG, "request %d: NULL sel / n_sel or empty capacity", r);
+      out[r] = PatchDesc{static_cast<uint8_t*>(reqs[r].kv_buf), static_cast<const uint8_t*>(reqs[r].fresh), s.sel, s.n_sel, reqs[r].T, s.sel_capacity};
+    }
+    return KVB_OK;
+  };
+  if (n_req <= kPatchInline && !c->force_copy) {  // the descriptors travel as the kernel's argument
+    PatchInline descs{};
+    const int f = fill(descs.d);
+    if (f != KVB_OK) return f;
+    c->last_stream = st;
+    KVB_CUDA(c, launch_patch_inline(descs, n_req, c->n_sm, c->dims, st));
+  } else {
+    uint8_t* host = nullptr;
+    const int slot_code = take_slot(c, &host);
+    if (slot_code >= 0) return slot_code;
+    const int slot = -slot_code - 1;
+    const int f = fill(reinterpret_cast<PatchDesc*>(host));
+    if (f != KVB_OK) return f;
+    const int up = upload(c, slot, host, sizeof(PatchDesc) * (size_t)n_req, st);
+    if (up != KVB_OK) return up;
+    c->last_stream = st;
+    KVB_CUDA(c, launch_patch_table(reinterpret_cast<const PatchDesc*>(c->arena_dev), n_req, c->n_sm, c->dims, st));
   }
-  const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req, st);
-  if (up != KVB_OK) return up;
-  c->last_stream = st;
-  KVB_CUDA(c, launch_patch(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, tiles, rows_per_cta, c->dims, st));
   c->launches += 1;
   return KVB_OK;
 }
@@ -700,8 +701,8 @@ int kvb_chunk_importance(kvb_ctx* c, const kvb_request* reqs, int n_req, float* 
   const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req, st);
   if (up != KVB_OK) return up;
   c->last_stream = st;
-  KVB_CUDA(c, launch_importance(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, chunks, c->dims, st));
-  c->launches += 1;
+  KVB_CUDA(c, launch_importance(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, chunks, c->dims, c->norm_sums, st));
+  c->launches += 2;
   return KVB_OK;
 }
 

@@ -52,6 +52,19 @@ struct ReqDesc {
   int32_t lhk_group;     // attention: (layer, head) pairs per scheduling group
 };
 
+struct PatchDesc {
+  uint8_t* kv_buf;
+  const uint8_t* fresh;
+  const int32_t* sel;
+  const int32_t* n_sel;
+  int32_t T;
+  int32_t sel_capacity;
+};
+constexpr int kPatchInline = 64;
+struct PatchInline {
+  PatchDesc d[kPatchInline];
+};
+
 struct SeamWindow {
   int32_t lo, hi;  // [lo, hi)
 };
@@ -111,9 +124,11 @@ cudaError_t attention_pair_configure();
 cudaError_t launch_attention_pair(const ReqDesc* reqs, const void* maps, int n_req, long long total_pairs, const ModelDims& m,
                                   float scale, uint32_t* status, int n_sm, bool pdl, cudaStream_t st);
 
-cudaError_t launch_patch(const ReqDesc* reqs, int n_req, int total_tiles, int rows_per_cta, const ModelDims& m,
-                         cudaStream_t st);
-cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, cudaStream_t st);
+// kvb_patch: one request's descriptor; up to kPatchInline of them travel as the kernel's own argument
+cudaError_t launch_patch_inline(const PatchInline& descs, int n_req, int n_sm, const ModelDims& m, cudaStream_t st);
+cudaError_t launch_patch_table(const PatchDesc* table, int n_req, int n_sm, const ModelDims& m, cudaStream_t st);
+// part: [total_chunks][L] doubles of scratch (the per-layer sums); two launches
+cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, double* part, cudaStream_t st);
 
 // One chunk to quantise (device memory).  k / v NULL: that side is not wanted.
 struct QuantJob {

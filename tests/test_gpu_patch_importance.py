@@ -16,8 +16,10 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-@pytest.mark.parametrize("idx,n_req", [(0, None), (4, 3)])
-def test_patch_matches_oracle(idx, n_req):
+@pytest.mark.parametrize("idx,n_req,table", [(0, None, False), (4, 3, False), (4, 3, True)])
+def test_patch_matches_oracle(idx, n_req, table):
+    """table: the descriptors go through the uploaded table (the route of calls with more requests than fit
+    the kernel's own argument) instead of travelling with the launch."""
     build_library()
     wl = synth.workload(idx, n_req) if n_req else synth.workload(idx)
     sh = wl.shape
@@ -27,6 +29,8 @@ def test_patch_matches_oracle(idx, n_req):
         tbl = run_assemble(ctx, reqs)
         sel, ks, caps = run_select(ctx, wl, reqs, tbl, use_oracle_buffer=False)
         before = [helpers.bits_of(r.kv_buf) for r in reqs]
+        if table:
+            B.kvb_set_debug_option(ctx, "descriptor_copy", 1)
         B.kvb_patch(ctx, tbl, sel)
         B.kvb_last_status(ctx)
         for i, r in enumerate(reqs):
