@@ -354,6 +354,8 @@ class Runner:
         ctx = B.create_for_shape(wl.shape, self.local, max_requests=len(wl.requests), max_chunks_total=n_chunks, max_tokens_total=n_tok)
         if args.attention_pairs:
             B.kvb_set_debug_option(ctx, "attention_cta_pairs", 1)
+        if args.attention_two_tiles:
+            B.kvb_set_debug_option(ctx, "attention_two_tiles", 1)
         n_rep = args.replicas or REPLICAS[key]
         reps = [Replica(B, ctx, wl, self.dev, 100 * self.rank + i, args.meta_fp16) for i in range(n_rep)]
         if key == "cfg3":  # the buffer and the selection the attention runs on, prepared outside the timed region
@@ -682,6 +684,8 @@ def main():
                     help="a K-step region shorter than this is repeated until this much device time has passed (0: one region, for profiler runs)")
     ap.add_argument("--attention-pairs", action="store_true",
                     help="run kvb_selective_attn in its paired-CTA form (the context's attention_cta_pairs option; measured slower, not the default)")
+    ap.add_argument("--attention-two-tiles", action="store_true",
+                    help="run kvb_selective_attn with two tiles per CTA sharing K/V (the context's attention_two_tiles option)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()

@@ -322,6 +322,10 @@ int64_t kvb_launch_count(kvb_ctx* ctx);
  *                                 sub-blocks of 128): measured slower than the default
  *                                 form, kept as a cross-check; same result to the
  *                                 attention tolerance, not bit for bit
+ *   "attention_two_tiles"         default 0; 1 runs kvb_selective_attn with two
+ *                                 neighbouring tiles per CTA that share every K/V
+ *                                 sub-block in shared memory, one CTA per SM; same
+ *                                 result to the attention tolerance
  * The first three settings compute the same bits; the tests compare them.
  * Unknown key or value: KVB_ERR_INVALID_ARG. */
 int kvb_set_debug_option(kvb_ctx* ctx, const char* key, int value);

@@ -44,6 +44,7 @@ struct kvb_ctx {
   bool force_copy = false;     // descriptors always go by cudaMemcpyAsync (cross-check)
   bool pdl = true;             // programmatic dependent launch along the kernel chain
   bool attn_pair = false;      // attention on CTA pairs (tcgen05 cta_group::2) instead of single CTAs
+  bool attn_dual = false;      // attention with two tiles per CTA sharing K/V, one CTA per SM
   cudaStream_t last_stream = nullptr;
   int64_t launches = 0;
   char err[512] = {0};
@@ -248,6 +249,7 @@ int kvb_create(kvb_ctx** out, int device, const kvb_model_desc* model, const kvb
   KVB_CUDA(c, topk_configure());
   KVB_CUDA(c, attention_tc_configure());
   KVB_CUDA(c, attention_pair_configure());
+  KVB_CUDA(c, attention_dual_configure());
   KVB_CUDA(c, quantize_configure());
 
   const int half = m.d / 2;
@@ -280,6 +282,7 @@ int kvb_set_debug_option(kvb_ctx* c, const char* key, int value) {
   else if (strcmp(key, "descriptor_copy") == 0) c->force_copy = value != 0;
   else if (strcmp(key, "attention_one_tile_per_cta") == 0) c->attn_one_tile = value != 0;
   else if (strcmp(key, "attention_cta_pairs") == 0) c->attn_pair = value != 0;
+  else if (strcmp(key, "attention_two_tiles") == 0) c->attn_dual = value != 0;
   else return fail(c, KVB_ERR_INVALID_ARG, "unknown debug option '%s'", key);
   return KVB_OK;
 }
@@ -612,7 +615,7 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
     }
     rd[r] = d;
     const int tiles_r = (s.sel_capacity + tok_per_tile - 1) / tok_per_tile;
-    tiles += c->attn_pair ? (tiles_r + 1) / 2 : tiles_r;  // the paired kernel counts pairs of neighbouring tiles
+    tiles += (c->attn_pair || c->attn_dual) ? (tiles_r + 1) / 2 : tiles_r;  // these kernels count pairs of neighbouring tiles
     const int e = attention_tc_encode_maps(c->dims, q[r], s.sel_capacity, reqs[r].kv_buf, reqs[r].T, host + maps_off + 256 * (size_t)r);
     if (e != 0) return fail(c, KVB_ERR_CUDA, "request %d: tensor map encoding failed (%d)", r, e);
   }
@@ -627,6 +630,9 @@ int kvb_selective_attn(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb
   if (c->attn_pair)
     KVB_CUDA(c, launch_attention_pair(rd_dev, c->arena_dev + maps_off, n_req, (long long)tiles * c->model.Hkv * c->model.L, c->dims,
                                       softmax_scale, c->status_dev, c->n_sm, c->pdl, st));
+  else if (c->attn_dual)
+    KVB_CUDA(c, launch_attention_dual(rd_dev, c->arena_dev + maps_off, n_req, tiles, c->dims, softmax_scale, c->status_dev,
+                                      reinterpret_cast<unsigned int*>(c->arena_dev + counter_off), c->n_sm, c->pdl, st));
   else
     KVB_CUDA(c, launch_attention_tc(rd_dev, c->arena_dev + maps_off, n_req, tiles, c->dims, softmax_scale, c->status_dev,
                                     reinterpret_cast<unsigned int*>(c->arena_dev + counter_off), c->n_sm, !c->attn_one_tile, c->pdl, st));

@@ -120,6 +120,10 @@ cudaError_t launch_attention_tc(const ReqDesc* reqs, const void* maps, int n_req
 
 // The paired form (csrc/attention_pair.cu): two tiles of one plane on two SMs per MMA.  total_pairs counts the
 // call's tile pairs over all requests and planes; ReqDesc::tile_offset counts a request's tile pairs per plane.
+// two neighbouring tiles per CTA, one CTA per SM (csrc/attention_dual.cu); tensor maps and tile counter as for the one-tile kernel
+cudaError_t attention_dual_configure();
+cudaError_t launch_attention_dual(const ReqDesc* reqs, const void* maps, int n_req, int total_pairs, const ModelDims& m, float scale,
+                                  uint32_t* status, unsigned int* tile_counter, int n_sm, bool pdl, cudaStream_t st);
 cudaError_t attention_pair_configure();
 cudaError_t launch_attention_pair(const ReqDesc* reqs, const void* maps, int n_req, long long total_pairs, const ModelDims& m,
                                   float scale, uint32_t* status, int n_sm, bool pdl, cudaStream_t st);

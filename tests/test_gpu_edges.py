@@ -373,8 +373,10 @@ def test_selection_cluster_path_plateaus_windows_and_extremes():
         B.kvb_destroy(ctx)
 
 
-def test_attention_cta_pair_form_matches_oracle():
-    """The paired form of the attention kernel (two neighbouring tiles on two SMs per MMA, the context's
+@pytest.mark.parametrize("option", ["attention_cta_pairs", "attention_two_tiles"])
+def test_attention_cta_pair_form_matches_oracle(option):
+    """(attention_two_tiles: two neighbouring tiles per CTA sharing K/V, one CTA per SM -- same check.)
+    The paired form of the attention kernel (two neighbouring tiles on two SMs per MMA, the context's
     "attention_cta_pairs" option; the single-CTA kernel is the default because it measures faster) computes
     the same attention: against the oracle at 2e-2 on a batch whose tiles are short, ragged, odd in number
     per plane and partly empty, with rows past n_sel left untouched.  Its bits may differ from the
@@ -386,7 +388,7 @@ def test_attention_cta_pair_form_matches_oracle():
     reqs = prepare(wl)
     ctx = B.create_for_shape(sh, 0, max_requests=len(reqs))
     try:
-        B.kvb_set_debug_option(ctx, "attention_cta_pairs", 1)
+        B.kvb_set_debug_option(ctx, option, 1)
         tbl = run_assemble(ctx, reqs)
         Ts = [r.plan.T for r in reqs]
         ks = [B.kvb_select_count(T, 0.2) for T in Ts]
@@ -394,7 +396,9 @@ def test_attention_cta_pair_form_matches_oracle():
         for r in reqs:
             r.sel_capacity = r.plan.T
         B.kvb_deviation_topk(ctx, tbl, 0.2, -1, 8, 8, 3, sel)
-        qs = [torch.randn(sh.L, T, sh.Hq, sh.d, device=DEV, generator=torch.Generator(DEV).manual_seed(T)).to(r.fresh.dtype) for T, r in zip(Ts, reqs)]
+        # queries by the workloads' recipe, N(0, 1 / d), for every row of the capacity
+        qs = [(torch.randn(sh.L, T, sh.Hq, sh.d, device=DEV, generator=torch.Generator(DEV).manual_seed(T)) / math.sqrt(sh.d)).to(r.fresh.dtype)
+              for T, r in zip(Ts, reqs)]
         out = [torch.zeros_like(q) for q in qs]
         for _ in range(2):
             B.kvb_selective_attn(ctx, tbl, sel, qs, out, 1.0 / math.sqrt(sh.d))
