@@ -48,6 +48,39 @@ def test_patch_matches_oracle(idx, n_req, table):
         B.kvb_destroy(ctx)
 
 
+@pytest.mark.parametrize("kv_dtype,Hkv,Hq", [("bf16", 1, 8), ("fp16", 8, 8), ("bf16", 4, 16)])
+def test_patch_other_row_widths(kv_dtype, Hkv, Hq):
+    """A token row of Hkv * 256 bytes is copied in 512-byte pieces, one warp each: half a warp for one KV
+    head, four pieces for eight.  Bit-exact against the oracle's row replacement; every other row untouched;
+    an out-of-range entry in the selection (a caller's stale list) is skipped."""
+    build_library()
+    sh = synth.Shape(L=3, Hq=Hq, Hkv=Hkv, kv_dtype=kv_dtype)
+    modes = [synth.MODE_INT8, synth.MODE_FRESH, synth.MODE_INT4, synth.MODE_INT8, synth.MODE_FP16]
+    wl = synth.Workload("patch", 41, sh, [synth._request(5 * sh.C, sh.C, modes, [512, 0, 128, 2048, 0]), synth._request(2 * sh.C, sh.C, modes[:2], [0, 0])],
+                        synth.SelectPlan(ratio=0.3, seam_before=4, seam_after=4))
+    reqs = prepare(wl)
+    ctx = B.create_for_shape(sh, 0)
+    try:
+        tbl = run_assemble(ctx, reqs)
+        sel, ks, caps = run_select(ctx, wl, reqs, tbl, use_oracle_buffer=False)
+        n0 = int(sel.n_sel[0])
+        good = sel.sel[0].cpu().numpy()[:n0].copy()
+        sel.sel[0][1] = reqs[0].plan.T + 5  # stale entries: beyond the prompt, negative
+        sel.sel[0][2] = -3
+        before = [helpers.bits_of(r.kv_buf) for r in reqs]
+        B.kvb_patch(ctx, tbl, sel)
+        B.kvb_last_status(ctx)
+        for i, r in enumerate(reqs):
+            n = int(sel.n_sel[i])
+            idxs = sel.sel[i].cpu().numpy()[:n]
+            if i == 0:
+                idxs = np.delete(good, [1, 2])
+            want = oracle.patch(before[i], helpers.bits_of(r.fresh), idxs)
+            assert np.array_equal(helpers.bits_of(r.kv_buf), want)
+    finally:
+        B.kvb_destroy(ctx)
+
+
 @pytest.mark.parametrize("kv_dtype,Hkv,Hq", [("bf16", 2, 16), ("fp16", 4, 8)])
 def test_chunk_importance_matches_oracle(kv_dtype, Hkv, Hq):
     build_library()
