@@ -612,8 +612,10 @@ class Runner:
             call = lambda rep: B.kvb_chunk_importance(ctx, rep.tbl, rep.imp)
             passage = "Eq. 7 (kvb_chunk_importance)"
         elif stage == "quantize":
-            # cache population of 128 chunks (a 16K-token prompt), keys and values, int8, one call
+            # cache population of 128 chunks (a 16K-token prompt), keys and values, one call
             n_jobs = 128
+            bits = args.quantize_bits
+            gk, gv = (1, 1) if bits == 8 else (sh.C // sh.int4_group, sh.d // sh.int4_group)  # groups per channel / per row
             g = torch.Generator(device=self.dev).manual_seed(5)
             for rep in reps:
                 rep.qjobs = []
@@ -621,15 +623,15 @@ class Runner:
                     kx = torch.randn((sh.L, sh.C, sh.Hkv, sh.d), generator=g, device=self.dev).to(sh.torch_dtype)
                     vx = torch.randn((sh.L, sh.C, sh.Hkv, sh.d), generator=g, device=self.dev).to(sh.torch_dtype)
                     mk = lambda *shape: torch.empty(shape, dtype=torch.uint8, device=self.dev)
-                    rep.qjobs.append(dict(k=kx, v=vx, k_codes=mk(sh.L, sh.C, sh.Hkv, sh.d), v_codes=mk(sh.L, sh.C, sh.Hkv, sh.d),
-                                          k_meta=torch.empty((sh.L, 1, sh.Hkv, sh.d, 2), device=self.dev),
-                                          v_meta=torch.empty((sh.L, sh.C, sh.Hkv, 1, 2), device=self.dev), bits=8))
+                    rep.qjobs.append(dict(k=kx, v=vx, k_codes=mk(sh.L, sh.C, sh.Hkv, sh.d * bits // 8), v_codes=mk(sh.L, sh.C, sh.Hkv, sh.d * bits // 8),
+                                          k_meta=torch.empty((sh.L, gk, sh.Hkv, sh.d, 2), device=self.dev),
+                                          v_meta=torch.empty((sh.L, sh.C, sh.Hkv, gv, 2), device=self.dev), bits=bits))
             E = sh.Hkv * sh.d
-            alg = n_jobs * sh.L * (2 * sh.C * E * 2 + 2 * sh.C * E + E * 8 + sh.C * sh.Hkv * 8)  # 16-bit rows read, codes and metadata written
+            alg = n_jobs * sh.L * (2 * sh.C * E * 2 + 2 * sh.C * E * bits // 8 + gk * E * 8 + sh.C * sh.Hkv * gv * 8)  # 16-bit rows read, codes and metadata written
             for rep in reps:
                 rep.qtable = B.QuantizeTable(rep.qjobs)  # marshalled once, like the request tables
             call = lambda rep: B.kvb_quantize_chunks(ctx, rep.qtable)
-            passage = "Eq. 6 forward (kvb_quantize_chunks), %d chunks x (keys + values), int8" % n_jobs
+            passage = "Eq. 6 forward (kvb_quantize_chunks), %d chunks x (keys + values), int%d" % (n_jobs, bits)
         else:
             raise SystemExit("unknown stage %s" % stage)
         for i in range(max(args.warmup, 3)):
@@ -684,6 +686,7 @@ def main():
                     help="a K-step region shorter than this is repeated until this much device time has passed (0: one region, for profiler runs)")
     ap.add_argument("--attention-pairs", action="store_true",
                     help="run kvb_selective_attn in its paired-CTA form (the context's attention_cta_pairs option; measured slower, not the default)")
+    ap.add_argument("--quantize-bits", type=int, default=8, choices=(4, 8), help="code width of --stage quantize")
     ap.add_argument("--attention-two-tiles", action="store_true",
                     help="run kvb_selective_attn with two tiles per CTA sharing K/V (the context's attention_two_tiles option)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
