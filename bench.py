@@ -545,7 +545,8 @@ class Runner:
                 s_cmp.wait_event(ev["in"])
 
         big = h2d + d2h > 4e9  # a step that moves tens of GB over PCIe takes about a second
-        n_warm, n_e2e = ((1, 3) if len(io) == 1 else (2, 4)) if big else (4, max(4, min(args.steps, 20)))
+        # pipelined steps: enough of them that filling and draining the two-deep pipeline weigh little
+        n_warm, n_e2e = ((1, 3) if len(io) == 1 else (2, 8)) if big else (4, max(4, min(args.steps, 20)))
         for i in range(n_warm):
             e2e_step(i)
         drain()
