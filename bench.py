@@ -626,13 +626,15 @@ class Runner:
                     mk = lambda *shape: torch.empty(shape, dtype=torch.uint8, device=self.dev)
                     rep.qjobs.append(dict(k=kx, v=vx, k_codes=mk(sh.L, sh.C, sh.Hkv, sh.d * bits // 8), v_codes=mk(sh.L, sh.C, sh.Hkv, sh.d * bits // 8),
                                           k_meta=torch.empty((sh.L, gk, sh.Hkv, sh.d, 2), device=self.dev),
-                                          v_meta=torch.empty((sh.L, sh.C, sh.Hkv, gv, 2), device=self.dev), bits=bits))
+                                          v_meta=torch.empty((sh.L, sh.C, sh.Hkv, gv, 2), device=self.dev), bits=bits,
+                                          unrotate_from=(sh.C * len(rep.qjobs) if args.quantize_unrotate else -1)))
             E = sh.Hkv * sh.d
             alg = n_jobs * sh.L * (2 * sh.C * E * 2 + 2 * sh.C * E * bits // 8 + gk * E * 8 + sh.C * sh.Hkv * gv * 8)  # 16-bit rows read, codes and metadata written
             for rep in reps:
                 rep.qtable = B.QuantizeTable(rep.qjobs)  # marshalled once, like the request tables
             call = lambda rep: B.kvb_quantize_chunks(ctx, rep.qtable)
-            passage = "Eq. 6 forward (kvb_quantize_chunks), %d chunks x (keys + values), int%d" % (n_jobs, bits)
+            passage = "Eq. 6 forward (kvb_quantize_chunks), %d chunks x (keys + values), int%d%s" % (
+                n_jobs, bits, ", keys rotated back to position 0 (Eq. 3)" if args.quantize_unrotate else "")
         else:
             raise SystemExit("unknown stage %s" % stage)
         for i in range(max(args.warmup, 3)):
@@ -688,6 +690,8 @@ def main():
     ap.add_argument("--attention-pairs", action="store_true",
                     help="run kvb_selective_attn in its paired-CTA form (the context's attention_cta_pairs option; measured slower, not the default)")
     ap.add_argument("--quantize-bits", type=int, default=8, choices=(4, 8), help="code width of --stage quantize")
+    ap.add_argument("--quantize-unrotate", action="store_true",
+                    help="--stage quantize: keys are rotated back from their positions first (position-free cache)")
     ap.add_argument("--attention-two-tiles", action="store_true",
                     help="run kvb_selective_attn with two tiles per CTA sharing K/V (the context's attention_two_tiles option)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
