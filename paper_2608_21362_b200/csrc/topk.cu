@@ -11,7 +11,8 @@
 // each owning a contiguous slice of the positions: every CTA counts its slice's histogram, sums all
 // CTAs' histograms through distributed shared memory and takes the same decision (one cluster
 // barrier per radix pass, histograms double-buffered); the prefix sums run locally, then over the
-// cluster; the first CTA gathers the winners and merge-sorts them.
+// cluster; every CTA sorts its own winners and ranks them against the other slices' sorted lists
+// (a merge sort in the first CTA remains for a slice that holds more winners than a CTA has threads).
 // The kernels are latency-bound (at most 128 KB of keys), so they are written to need few barriers:
 // warp-aggregated histogram updates, one combined prefix sum for the selection, conflict-free
 // shared-memory access.
@@ -80,6 +81,37 @@ __device__ __forceinline__ unsigned long long ce_step(unsigned long long v, int 
   const unsigned long long o = shfl_xor64(v, stride);
   const bool take_min = ((lane & stride) == 0) == up;
   return take_min ? (v < o ? v : o) : (v > o ? v : o);
+}
+
+// Ascending bitonic sort of n_pad values (a power of two, 32 .. kThreads), one per thread tid < n_pad,
+// held in a register for the whole sort.  Strides below 32 are shuffles; larger strides publish the
+// element and read the partner's, alternating between buf0 and buf1 so that one barrier per step is
+// enough.  Only the n_pad threads that hold an element take part (named barrier 1); whole warps.
+__device__ __forceinline__ unsigned long long block_bitonic_sort(unsigned long long v, int n_pad, int tid, int lane,
+                                                                 unsigned long long* buf0, unsigned long long* buf1) {
+#pragma unroll
+  for (int size = 2; size <= 32; size <<= 1) {
+    const bool up = (tid & size) == 0;
+#pragma unroll
+    for (int stride = size >> 1; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+  }
+  unsigned long long* bufs[2] = {buf0, buf1};
+  int b = 0;
+  for (int size = 64; size <= n_pad; size <<= 1) {
+    const bool up = (tid & size) == 0;
+    for (int stride = size >> 1; stride >= 32; stride >>= 1) {
+      bufs[b][tid] = v;
+      asm volatile("bar.sync 1, %0;" ::"r"(n_pad) : "memory");
+      const unsigned long long o = bufs[b][tid ^ stride];
+      const bool take_min = ((tid & stride) == 0) == up;
+      v = take_min ? (v < o ? v : o) : (v > o ? v : o);
+      b ^= 1;
+    }
+#pragma unroll
+    for (int stride = 16; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+  }
+  if (n_pad >= 64) asm volatile("bar.sync 1, %0;" ::"r"(n_pad) : "memory");  // the last partner reads are done
+  return v;
 }
 
 // One CTA per request: the form for prompts of up to kSplitTokens positions, where a cluster's
@@ -359,12 +391,14 @@ __global__ void __launch_bounds__(kThreads, 1)
                         unsigned long long* __restrict__ acc, int slice_pad, int k_pad, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
   // dynamic: keys of the slice; inverted keys and positions of the slice's winners (index order);
-  // two buffers for the merge sort of the request's winners (ranking CTA only)
+  // two buffers for the request's winners (all slices' sorted lists side by side; the merge sort of
+  // the fallback); two buffers for the sort of this slice's winners
   const int loc_pad = slice_pad < k_pad ? slice_pad : k_pad;
   uint32_t* s_keys = reinterpret_cast<uint32_t*>(smem);  // [slice_pad]
   uint32_t* s_lkey = s_keys + slice_pad;                 // [loc_pad]
   uint32_t* s_lidx = s_lkey + loc_pad;                   // [loc_pad]
   unsigned long long* s_grp = reinterpret_cast<unsigned long long*>(s_lidx + loc_pad);  // 2 x [k_pad rounded up to 32]
+  unsigned long long* s_sort = s_grp + 2 * ((k_pad + 31) & ~31);  // 2 x [kThreads]: this slice's winners, sorted (read by the other CTAs)
   __shared__ Shared sh;
   __shared__ uint32_t s_tot[256];          // histogram summed over the cluster
   __shared__ uint32_t s_warp_sums[33];
@@ -601,12 +635,62 @@ __global__ void __launch_bounds__(kThreads, 1)
     if (n_all != (uint32_t)k) atomicOr(status, DEV_STATUS_BAD_DESC);
   }
 
-  // ---- 5. rank, by the first CTA of the cluster: a merge sort of the winners' composite values
-  //      (inverted key, index), ascending = key descending, index ascending.  Runs of 32 are sorted by
-  //      a bitonic network in registers (one element per lane), then runs are merged pairwise: every
-  //      element finds its place in the merged run by a binary search of the sibling run.  All values
-  //      are distinct; the padding (all ones) sorts last and the merge keeps equal values in run order.
-  if (c == 0 && n_all == (uint32_t)k && k > 0) {
+  // ---- 5. rank: the winners' composite values (inverted key, index) in ascending order = key
+  //      descending, index ascending.  Every CTA sorts its slice's winners (one per thread, bitonic
+  //      network in registers); after a cluster barrier it copies all slices' sorted lists into its own
+  //      shared memory and each of its winners finds, by a binary search per other list, how many
+  //      winners of the other slices precede it: own place + those counts = its rank.  All values are
+  //      distinct.  The same in every CTA of the cluster: whether every slice's list fits a CTA.
+  bool spread = n_all == (uint32_t)k && k > 0;
+#pragma unroll
+  for (int r = 0; r < kMaxCluster; ++r) spread = spread && win_r[r] <= (uint32_t)kThreads;
+  if (spread) {
+    int n_pad = 32;
+    while (n_pad < (int)n_win) n_pad <<= 1;
+    unsigned long long v = ~0ull;  // padding sorts last
+    if (tid < (int)n_win) v = ((unsigned long long)s_lkey[tid] << 32) | s_lidx[tid];
+    if (tid < n_pad) {
+      v = block_bitonic_sort(v, n_pad, tid, lane, s_sort, s_sort + kThreads);
+      s_sort[tid] = v;
+    }
+    cluster_barrier();  // every slice's sorted list is complete
+    uint32_t off_r[kMaxCluster];
+    {
+      uint32_t o = 0;
+#pragma unroll
+      for (int r = 0; r < kMaxCluster; ++r) {
+        off_r[r] = o;
+        o += win_r[r];
+      }
+    }
+    for (uint32_t e = tid; e < n_all; e += kThreads) {  // entry e of the side-by-side lists is entry e - off_r of slice r's
+      int r = 0;
+#pragma unroll
+      for (int rr = 1; rr < kMaxCluster; ++rr)
+        if (rr < S && e >= off_r[rr]) r = rr;
+      s_grp[e] = cluster.map_shared_rank(s_sort, r)[e - off_r[r]];
+    }
+    __syncthreads();
+    if (tid < (int)n_win) {
+      uint32_t place = (uint32_t)tid;
+#pragma unroll
+      for (int r = 0; r < kMaxCluster; ++r) {
+        if (r >= S || r == c) continue;
+        const unsigned long long* a = s_grp + off_r[r];
+        uint32_t lo = 0, hi = win_r[r];  // entries of slice r below v
+        while (lo < hi) {
+          const uint32_t mid = (lo + hi) >> 1;
+          if (a[mid] < v) lo = mid + 1; else hi = mid;
+        }
+        place += lo;
+      }
+      rq.rank[place] = (int32_t)(uint32_t)(v & 0xFFFFFFFFull);
+    }
+  } else if (c == 0 && n_all == (uint32_t)k && k > 0) {
+    // fallback (a slice with more winners than threads), by the first CTA: a merge sort.  Runs of 32 are
+    // sorted by a bitonic network in registers (one element per lane), then runs are merged pairwise:
+    // every element finds its place in the merged run by a binary search of the sibling run; the
+    // padding (all ones) sorts last and the merge keeps equal values in run order.
     constexpr int kPer = kMaxK / kThreads;  // elements per thread
     const uint32_t n_pad = (n_all + 31u) & ~31u;
     unsigned long long *src = s_grp, *dst = s_grp + ((k_pad + 31) & ~31);
@@ -680,7 +764,7 @@ int cluster_size(int max_T) {
 
 size_t cluster_smem(int slice_pad, int k_pad) {
   const size_t loc = (size_t)(slice_pad < k_pad ? slice_pad : k_pad);
-  return (size_t)slice_pad * 4 + loc * 8 + (size_t)((k_pad + 31) & ~31) * 16;
+  return (size_t)slice_pad * 4 + loc * 8 + (size_t)((k_pad + 31) & ~31) * 16 + (size_t)kThreads * 16;
 }
 
 size_t single_smem(int t_pad, int k_pad) { return (size_t)t_pad * 4 + kThreads * 4 + (size_t)(k_pad < 32 ? 32 : k_pad) * 8; }
