@@ -6,8 +6,9 @@
 //   3. the k winners sorted in that order -> rank;
 //   4. bitmask union with the seam windows, prefix sums -> ascending sel and n_sel.
 // All decisions are integer comparisons: the result is a pure function of the float32 delta.
-// Two kernels.  Prompts of up to 2048 positions take one CTA per request (a bitonic network sorts the
-// winners, one per thread).  Longer prompts take a thread-block cluster of up to 8 CTAs per request,
+// Two kernels.  Prompts of up to 2048 positions take one CTA per request (warps sort runs of 32
+// winners and every winner is ranked against the other runs by binary searches).  Longer prompts
+// take a thread-block cluster of up to 8 CTAs per request,
 // each owning a contiguous slice of the positions: every CTA counts its slice's histogram, sums all
 // CTAs' histograms through distributed shared memory and takes the same decision (one cluster
 // barrier per radix pass, histograms double-buffered); the prefix sums run locally, then over the
@@ -85,35 +86,39 @@ __device__ __forceinline__ unsigned long long ce_step(unsigned long long v, int 
   return take_min ? (v < o ? v : o) : (v > o ? v : o);
 }
 
-// Ascending bitonic sort of n_pad values (a power of two, 32 .. kThreads), one per thread tid < n_pad,
-// held in a register for the whole sort.  Strides below 32 are shuffles; larger strides publish the
-// element and read the partner's, alternating between buf0 and buf1 so that one barrier per step is
-// enough.  Only the n_pad threads that hold an element take part (named barrier 1); whole warps.
-__device__ __forceinline__ unsigned long long block_bitonic_sort(unsigned long long v, int n_pad, int tid, int lane,
-                                                                 unsigned long long* buf0, unsigned long long* buf1) {
+// Ranks n <= kThreads distinct values, value i held by thread i (v; threads beyond n pass anything):
+// every warp sorts a run of 32 of them (one per lane, bitonic network in registers) into
+// runs[32 w .. 32 w + 31], padded with all ones, then each value finds by a binary search per other
+// run how many of that run's values precede it; own place in the run + those counts = its rank.
+// On return v is the value this thread holds after its warp's sort and the result is its rank (only
+// meaningful when v is not the padding).  Contains a block-wide barrier: every thread calls it.
+__device__ __forceinline__ uint32_t rank_by_runs(unsigned long long& v, int n, int tid, int lane, int warp, unsigned long long* runs) {
+  const int n_runs = (n + 31) >> 5;
+  if (tid >= n) v = ~0ull;
+  if (warp < n_runs) {
 #pragma unroll
-  for (int size = 2; size <= 32; size <<= 1) {
-    const bool up = (tid & size) == 0;
+    for (int size = 2; size <= 32; size <<= 1) {
+      const bool up = (lane & size) == 0 || size == 32;  // the last stage leaves the run ascending
 #pragma unroll
-    for (int stride = size >> 1; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
-  }
-  unsigned long long* bufs[2] = {buf0, buf1};
-  int b = 0;
-  for (int size = 64; size <= n_pad; size <<= 1) {
-    const bool up = (tid & size) == 0;
-    for (int stride = size >> 1; stride >= 32; stride >>= 1) {
-      bufs[b][tid] = v;
-      asm volatile("bar.sync 1, %0;" ::"r"(n_pad) : "memory");
-      const unsigned long long o = bufs[b][tid ^ stride];
-      const bool take_min = ((tid & stride) == 0) == up;
-      v = take_min ? (v < o ? v : o) : (v > o ? v : o);
-      b ^= 1;
+      for (int stride = size >> 1; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
     }
-#pragma unroll
-    for (int stride = 16; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
+    runs[tid] = v;
   }
-  if (n_pad >= 64) asm volatile("bar.sync 1, %0;" ::"r"(n_pad) : "memory");  // the last partner reads are done
-  return v;
+  __syncthreads();
+  uint32_t place = (uint32_t)lane;
+  if (warp < n_runs && v != ~0ull) {
+    for (int r = 0; r < n_runs; ++r) {
+      if (r == warp) continue;
+      const unsigned long long* run = runs + (r << 5);
+      uint32_t lo = 0;  // entries of run r below v
+#pragma unroll
+      for (int step = 16; step > 0; step >>= 1)
+        if (run[lo + step - 1] < v) lo += step;
+      if (run[lo] < v) ++lo;  // lo <= 31 here
+      place += lo;
+    }
+  }
+  return place;
 }
 
 // One CTA per request: the form for prompts of up to kSingleTokens positions, where a cluster's
@@ -257,40 +262,15 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
   __syncthreads();
 
-  // ---- bitonic sort of s_comp[0..k_pad): element i lives in lane i % 32 of its warp for the steps
-  //      with stride < 32 (registers + shuffles); larger strides go through shared memory
-  if (k_pad >= 64 && k_pad <= kThreads && (size_t)k_pad * 8 <= (size_t)t_pad * 4) {
-    // One element per thread, held in a register for the whole sort.  Strides below 32 are shuffles;
-    // larger strides publish the element and read the partner's, alternating between s_comp and the
-    // key array (no longer needed) so that one barrier per step is enough.  Only the k_pad threads
-    // that hold an element take part (named barrier 1).
-    if (tid < k_pad) {
-      unsigned long long* bufs[2] = {s_comp, reinterpret_cast<unsigned long long*>(s_keys)};
-      unsigned long long v = s_comp[tid];
-#pragma unroll
-      for (int size = 2; size <= 32; size <<= 1) {
-        const bool up = (tid & size) == 0;
-#pragma unroll
-        for (int stride = size >> 1; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
-      }
-      int b = 1;
-      for (int size = 64; size <= k_pad; size <<= 1) {
-        const bool up = (tid & size) == 0;
-        for (int stride = size >> 1; stride >= 32; stride >>= 1) {
-          bufs[b][tid] = v;
-          asm volatile("bar.sync 1, %0;" ::"r"(k_pad) : "memory");
-          const unsigned long long o = bufs[b][tid ^ stride];
-          const bool take_min = ((tid & stride) == 0) == up;
-          v = take_min ? (v < o ? v : o) : (v > o ? v : o);
-          b ^= 1;
-        }
-#pragma unroll
-        for (int stride = 16; stride > 0; stride >>= 1) v = ce_step(v, lane, stride, up);
-      }
-      asm volatile("bar.sync 1, %0;" ::"r"(k_pad) : "memory");  // the last partner reads are done
-      s_comp[tid] = v;
-    }
-    __syncthreads();
+  // ---- rank.  Up to kThreads winners: runs of 32 sorted by the warps, every winner ranked against the
+  //      other runs (rank_by_runs), its position written at once.
+  bool ranked = false;
+  if (k_pad >= 64 && k_pad <= kThreads) {
+    unsigned long long v = tid < k ? s_comp[tid] : ~0ull;
+    __syncthreads();  // s_comp becomes the runs
+    const uint32_t place = rank_by_runs(v, k, tid, lane, warp, s_comp);
+    if (v != ~0ull) rq.rank[place] = (int32_t)(uint32_t)(v & 0xFFFFFFFFull);
+    ranked = true;
   } else if (k_pad >= 32) {
     for (int i0 = 0; i0 < k_pad; i0 += kThreads) {  // sizes 2..32 entirely in registers
       const int i = i0 + tid;
@@ -343,7 +323,8 @@ __global__ void __launch_bounds__(kThreads, 1)
     }
     __syncthreads();
   }
-  for (int i = tid; i < k; i += kThreads) rq.rank[i] = (int32_t)(uint32_t)(s_comp[i] & 0xFFFFFFFFull);
+  if (!ranked)
+    for (int i = tid; i < k; i += kThreads) rq.rank[i] = (int32_t)(uint32_t)(s_comp[i] & 0xFFFFFFFFull);
 
   // ---- 4. union with the seam windows, ascending list
   //      (a warp per window, a lane per mask word of the window)
@@ -638,8 +619,8 @@ __global__ void __launch_bounds__(kThreads, 1)
   }
 
   // ---- 5. rank: the winners' composite values (inverted key, index) in ascending order = key
-  //      descending, index ascending.  Every CTA sorts its slice's winners (one per thread, bitonic
-  //      network in registers); after a cluster barrier it copies all slices' sorted lists into its own
+  //      descending, index ascending.  Every CTA sorts its slice's winners (rank_by_runs, then each
+  //      value stored at its place); after a cluster barrier it copies all slices' sorted lists into its own
   //      shared memory and each of its winners finds, by a binary search per other list, how many
   //      winners of the other slices precede it: own place + those counts = its rank.  All values are
   //      distinct.  The same in every CTA of the cluster: whether every slice's list fits a CTA.
@@ -647,14 +628,10 @@ __global__ void __launch_bounds__(kThreads, 1)
 #pragma unroll
   for (int r = 0; r < kMaxCluster; ++r) spread = spread && win_r[r] <= (uint32_t)kThreads;
   if (spread) {
-    int n_pad = 32;
-    while (n_pad < (int)n_win) n_pad <<= 1;
-    unsigned long long v = ~0ull;  // padding sorts last
+    unsigned long long v = ~0ull;
     if (tid < (int)n_win) v = ((unsigned long long)s_lkey[tid] << 32) | s_lidx[tid];
-    if (tid < n_pad) {
-      v = block_bitonic_sort(v, n_pad, tid, lane, s_sort, s_sort + kThreads);
-      s_sort[tid] = v;
-    }
+    const uint32_t local_place = rank_by_runs(v, (int)n_win, tid, lane, warp, s_sort + kThreads);
+    if (v != ~0ull) s_sort[local_place] = v;  // this slice's winners in ascending order
     cluster_barrier();  // every slice's sorted list is complete
     uint32_t off_r[kMaxCluster];
     {
@@ -673,8 +650,8 @@ __global__ void __launch_bounds__(kThreads, 1)
       s_grp[e] = cluster.map_shared_rank(s_sort, r)[e - off_r[r]];
     }
     __syncthreads();
-    if (tid < (int)n_win) {
-      uint32_t place = (uint32_t)tid;
+    if (v != ~0ull) {
+      uint32_t place = local_place;
 #pragma unroll
       for (int r = 0; r < kMaxCluster; ++r) {
         if (r >= S || r == c) continue;
