@@ -8,6 +8,7 @@
 
 #include "f32x2.cuh"
 #include "kvb_internal.h"
+#include "pdl.cuh"
 
 namespace kvb {
 namespace {
@@ -64,9 +65,11 @@ __device__ __forceinline__ void patch_body(Fetch fetch, int n_req, const ModelDi
 }
 
 __global__ void __launch_bounds__(kThreads) patch_inline_kernel(const __grid_constant__ PatchInline a, int n_req, ModelDims m) {
+  pdl_wait();  // the selection (and the table) come from the kernels before this one
   patch_body([&](int r) { return a.d[r]; }, n_req, m);
 }
 __global__ void __launch_bounds__(kThreads) patch_table_kernel(const PatchDesc* __restrict__ table, int n_req, ModelDims m) {
+  pdl_wait();
   patch_body([&](int r) { return table[r]; }, n_req, m);
 }
 
@@ -88,6 +91,7 @@ __global__ void __launch_bounds__(kThreads)
   constexpr int kUnroll = 4;
   __shared__ double s_part[kThreads / 32];
   const int item = blockIdx.x, l = blockIdx.y;
+  pdl_wait();  // the table and the buffer come from the kernels before this one
   const ReqDesc rq = reqs[request_of(reqs, n_req, item)];
   const int chunk = item - rq.tile_offset;
   const int H = m.Hkv, C = m.C;
@@ -139,6 +143,7 @@ __global__ void __launch_bounds__(kThreads)
 __global__ void importance_mean_kernel(const ReqDesc* __restrict__ reqs, int n_req, int total_chunks, ModelDims m,
                                        const double* __restrict__ part) {
   const int item = blockIdx.x * blockDim.x + threadIdx.x;
+  pdl_wait();
   if (item >= total_chunks) return;
   const ReqDesc rq = reqs[request_of(reqs, n_req, item)];
   double tot = 0.0;
@@ -148,24 +153,21 @@ __global__ void importance_mean_kernel(const ReqDesc* __restrict__ reqs, int n_r
 
 }  // namespace
 
-cudaError_t launch_patch_inline(const PatchInline& descs, int n_req, int n_sm, const ModelDims& m, cudaStream_t st) {
-  patch_inline_kernel<<<(unsigned)(n_sm * kPatchCtasPerSm), kThreads, 0, st>>>(descs, n_req, m);
-  return cudaGetLastError();
+cudaError_t launch_patch_inline(const PatchInline& descs, int n_req, int n_sm, const ModelDims& m, bool pdl, cudaStream_t st) {
+  return launch_pdl(pdl, patch_inline_kernel, dim3((unsigned)(n_sm * kPatchCtasPerSm)), dim3(kThreads), 0, st, descs, n_req, m);
 }
 
-cudaError_t launch_patch_table(const PatchDesc* table, int n_req, int n_sm, const ModelDims& m, cudaStream_t st) {
-  patch_table_kernel<<<(unsigned)(n_sm * kPatchCtasPerSm), kThreads, 0, st>>>(table, n_req, m);
-  return cudaGetLastError();
+cudaError_t launch_patch_table(const PatchDesc* table, int n_req, int n_sm, const ModelDims& m, bool pdl, cudaStream_t st) {
+  return launch_pdl(pdl, patch_table_kernel, dim3((unsigned)(n_sm * kPatchCtasPerSm)), dim3(kThreads), 0, st, table, n_req, m);
 }
 
-cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, double* part, cudaStream_t st) {
+cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, double* part, bool pdl, cudaStream_t st) {
   const dim3 grid((unsigned)total_chunks, (unsigned)m.L);
-  if (m.dtype == KVB_DT_BF16)
-    importance_kernel<KVB_DT_BF16><<<grid, kThreads, 0, st>>>(reqs, n_req, m, part);
-  else
-    importance_kernel<KVB_DT_F16><<<grid, kThreads, 0, st>>>(reqs, n_req, m, part);
-  importance_mean_kernel<<<(total_chunks + 127) / 128, 128, 0, st>>>(reqs, n_req, total_chunks, m, part);
-  return cudaGetLastError();
+  cudaError_t e = m.dtype == KVB_DT_BF16 ? launch_pdl(pdl, importance_kernel<KVB_DT_BF16>, grid, dim3(kThreads), 0, st, reqs, n_req, m, part)
+                                         : launch_pdl(pdl, importance_kernel<KVB_DT_F16>, grid, dim3(kThreads), 0, st, reqs, n_req, m, part);
+  if (e != cudaSuccess) return e;
+  return launch_pdl(pdl, importance_mean_kernel, dim3((unsigned)((total_chunks + 127) / 128)), dim3(128), 0, st, reqs, n_req, total_chunks, m,
+                    static_cast<const double*>(part));
 }
 
 }  // namespace kvb

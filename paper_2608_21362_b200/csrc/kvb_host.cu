@@ -662,7 +662,7 @@ int kvb_patch(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_selectio
     const int f = fill(descs.d);
     if (f != KVB_OK) return f;
     c->last_stream = st;
-    KVB_CUDA(c, launch_patch_inline(descs, n_req, c->n_sm, c->dims, st));
+    KVB_CUDA(c, launch_patch_inline(descs, n_req, c->n_sm, c->dims, c->pdl, st));
   } else {
     uint8_t* host = nullptr;
     const int slot_code = take_slot(c, &host);
@@ -673,7 +673,7 @@ int kvb_patch(kvb_ctx* c, const kvb_request* reqs, int n_req, const kvb_selectio
     const int up = upload(c, slot, host, sizeof(PatchDesc) * (size_t)n_req, st);
     if (up != KVB_OK) return up;
     c->last_stream = st;
-    KVB_CUDA(c, launch_patch_table(reinterpret_cast<const PatchDesc*>(c->arena_dev), n_req, c->n_sm, c->dims, st));
+    KVB_CUDA(c, launch_patch_table(reinterpret_cast<const PatchDesc*>(c->arena_dev), n_req, c->n_sm, c->dims, c->pdl, st));
   }
   c->launches += 1;
   return KVB_OK;
@@ -707,7 +707,7 @@ int kvb_chunk_importance(kvb_ctx* c, const kvb_request* reqs, int n_req, float* 
   const int up = upload(c, slot, host, sizeof(ReqDesc) * (size_t)n_req, st);
   if (up != KVB_OK) return up;
   c->last_stream = st;
-  KVB_CUDA(c, launch_importance(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, chunks, c->dims, c->norm_sums, st));
+  KVB_CUDA(c, launch_importance(reinterpret_cast<const ReqDesc*>(c->arena_dev), n_req, chunks, c->dims, c->norm_sums, c->pdl, st));
   c->launches += 2;
   return KVB_OK;
 }
@@ -743,7 +743,7 @@ int kvb_quantize_chunks(kvb_ctx* c, const kvb_quantize_job* jobs, int n_jobs, vo
   const int up = upload(c, slot, host, sizeof(QuantJob) * (size_t)n_jobs, st);
   if (up != KVB_OK) return up;
   c->last_stream = st;
-  KVB_CUDA(c, launch_quantize_batch(reinterpret_cast<const QuantJob*>(c->arena_dev), n_jobs, c->dims, c->inv_freq, c->status_dev, st));
+  KVB_CUDA(c, launch_quantize_batch(reinterpret_cast<const QuantJob*>(c->arena_dev), n_jobs, c->dims, c->inv_freq, c->status_dev, c->pdl, st));
   c->launches += 1;
   return KVB_OK;
 }

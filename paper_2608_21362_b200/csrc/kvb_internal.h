@@ -129,10 +129,10 @@ cudaError_t launch_attention_pair(const ReqDesc* reqs, const void* maps, int n_r
                                   float scale, uint32_t* status, int n_sm, bool pdl, cudaStream_t st);
 
 // kvb_patch: one request's descriptor; up to kPatchInline of them travel as the kernel's own argument
-cudaError_t launch_patch_inline(const PatchInline& descs, int n_req, int n_sm, const ModelDims& m, cudaStream_t st);
-cudaError_t launch_patch_table(const PatchDesc* table, int n_req, int n_sm, const ModelDims& m, cudaStream_t st);
+cudaError_t launch_patch_inline(const PatchInline& descs, int n_req, int n_sm, const ModelDims& m, bool pdl, cudaStream_t st);
+cudaError_t launch_patch_table(const PatchDesc* table, int n_req, int n_sm, const ModelDims& m, bool pdl, cudaStream_t st);
 // part: [total_chunks][L] doubles of scratch (the per-layer sums); two launches
-cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, double* part, cudaStream_t st);
+cudaError_t launch_importance(const ReqDesc* reqs, int n_req, int total_chunks, const ModelDims& m, double* part, bool pdl, cudaStream_t st);
 
 // One chunk to quantise (device memory).  k / v NULL: that side is not wanted.
 struct QuantJob {
@@ -149,7 +149,7 @@ struct QuantJob {
 };
 // inv_freq: [d/2] doubles, device
 cudaError_t launch_quantize_batch(const QuantJob* jobs, int n_jobs, const ModelDims& m, const double* inv_freq,
-                                  uint32_t* status, cudaStream_t st);
+                                  uint32_t* status, bool pdl, cudaStream_t st);
 cudaError_t quantize_configure();
 
 }  // namespace kvb

@@ -28,6 +28,7 @@
 #include <type_traits>
 
 #include "kvb_internal.h"
+#include "pdl.cuh"
 
 namespace kvb {
 namespace {
@@ -236,6 +237,7 @@ __global__ void __launch_bounds__(kThreads, 3)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int H = m.Hkv;
   const int n_hp = H / HP;
+  pdl_wait();  // the job table comes from the kernel before this one
   int item = blockIdx.x;
   const int hb = (item % n_hp) * HP;      // first head
   item /= n_hp;
@@ -583,18 +585,16 @@ cudaError_t quantize_configure() {
 }
 
 cudaError_t launch_quantize_batch(const QuantJob* jobs, int n_jobs, const ModelDims& m, const double* inv_freq, uint32_t* status,
-                                  cudaStream_t st) {
+                                  bool pdl, cudaStream_t st) {
   const int hp = m.Hkv < 2 ? 1 : 2;
-  const unsigned grid = (unsigned)n_jobs * m.L * 2 * (m.Hkv / hp);
+  const dim3 grid((unsigned)n_jobs * m.L * 2 * (m.Hkv / hp)), block(kThreads);
   const bool bf16 = m.dtype == KVB_DT_BF16;
   if (hp == 2) {
-    if (bf16) quantize_batch_kernel<KVB_DT_BF16, 2><<<grid, kThreads, quantize_smem(2), st>>>(jobs, m, inv_freq, status);
-    else quantize_batch_kernel<KVB_DT_F16, 2><<<grid, kThreads, quantize_smem(2), st>>>(jobs, m, inv_freq, status);
-  } else {
-    if (bf16) quantize_batch_kernel<KVB_DT_BF16, 1><<<grid, kThreads, quantize_smem(1), st>>>(jobs, m, inv_freq, status);
-    else quantize_batch_kernel<KVB_DT_F16, 1><<<grid, kThreads, quantize_smem(1), st>>>(jobs, m, inv_freq, status);
+    if (bf16) return launch_pdl(pdl, quantize_batch_kernel<KVB_DT_BF16, 2>, grid, block, quantize_smem(2), st, jobs, m, inv_freq, status);
+    return launch_pdl(pdl, quantize_batch_kernel<KVB_DT_F16, 2>, grid, block, quantize_smem(2), st, jobs, m, inv_freq, status);
   }
-  return cudaGetLastError();
+  if (bf16) return launch_pdl(pdl, quantize_batch_kernel<KVB_DT_BF16, 1>, grid, block, quantize_smem(1), st, jobs, m, inv_freq, status);
+  return launch_pdl(pdl, quantize_batch_kernel<KVB_DT_F16, 1>, grid, block, quantize_smem(1), st, jobs, m, inv_freq, status);
 }
 
 }  // namespace kvb
