@@ -193,7 +193,8 @@ int kvb_selective_attn(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const k
  * SelectiveRecompute (Algorithm 1): for every request and every i < *n_sel,
  * the K and V rows of position sel[i] in every layer of kv_buf are replaced
  * by the rows of `fresh` (K~, V~).  sel: host array of n_req kvb_selection
- * (only sel, n_sel, sel_capacity are read).  Other rows are not touched. */
+ * (only sel, n_sel, sel_capacity are read).  Other rows are not touched; an
+ * entry of sel outside [0, T) is skipped. */
 int kvb_patch(kvb_ctx* ctx, const kvb_request* reqs, int n_req, const kvb_selection* sel, void* cuda_stream);
 
 /* Importance score of the cache manager's eviction policy (KV Cache Manager,
